@@ -1,0 +1,223 @@
+"""Pins for the oracle's decode procedure: the invariants the paper's method implies."""
+import itertools
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from oracle import tidar_oracle as O
+from tidar_synth import CONFIGS, gen_model_weights, gen_token_ids, tensor_id
+
+
+def _cfg(sh, beta=1.0):
+    return O.OracleConfig(sh.n_layers, sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.d_ffn,
+                          sh.vocab, sh.rope_theta, sh.rms_eps, sh.mask_token_id, beta)
+
+
+@pytest.fixture(scope="module", params=["tied", "untied"])
+def model(request):
+    # the tied tiny model repeats one token under random weights; the untied twin
+    # wanders, so both degenerate and non-degenerate sequences are covered
+    sh = replace(CONFIGS["tiny"], tie_lm_head=(request.param == "tied"))
+    w = O.weights_to_f64(gen_model_weights(sh))
+    prompt = gen_token_ids(sh.seed, tensor_id("prompt"), sh.prompt_len, sh.vocab - 1).numpy().astype(np.int64)
+    return sh, _cfg(sh), w, prompt
+
+
+N_NEW = 24
+
+
+@pytest.fixture(scope="module")
+def ar_tokens(model):
+    sh, cfg, w, prompt = model
+    return O.ar_generate(cfg, w, prompt, N_NEW + 2 * sh.k)
+
+
+# ---------------------------------------------------------------- acceptance rule
+def _accept_brute(block, targets):
+    k = len(block)
+    best = 0
+    for m in range(k):
+        if all(block[i] == targets[i - 1] for i in range(1, m + 1)):
+            best = max(best, m)
+    return best + 1
+
+
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_accept_length_exhaustive(k):
+    targets = list(range(100, 100 + k))
+    for pattern in itertools.product([True, False], repeat=k - 1):
+        block = [7] + [targets[i] if ok else -1 for i, ok in enumerate(pattern)]
+        L = O.accept_length(block, targets)
+        assert L == _accept_brute(block, targets)
+        assert 1 <= L <= k
+        first_bad = next((i for i, ok in enumerate(pattern) if not ok), k - 1)
+        assert L == first_bad + 1
+
+
+def test_accept_forced_and_select():
+    block = [5, 6, 7, 8]
+    targets = [6, 9, 9, 9]
+    assert O.accept_length(block, targets) == 2
+    assert O.accept_length(block, targets, forced=4) == 4
+    d = np.arange(16).reshape(4, 4) + 100
+    np.testing.assert_array_equal(O.select_next(2, targets, d), [9, 105, 106, 107])
+
+
+# ---------------------------------------------------------------- greedy TiDAR == greedy AR
+def test_tidar_equals_ar_natural_drafts(model, ar_tokens):
+    sh, cfg, w, prompt = model
+    out, Ls, _ = O.generate(cfg, w, prompt, sh.k, N_NEW)
+    assert out == ar_tokens[:N_NEW]
+    assert all(1 <= L <= sh.k for L in Ls)
+
+
+def test_tidar_equals_ar_garbage_drafts(model, ar_tokens):
+    sh, cfg, w, prompt = model
+
+    def hook(st):                      # drafts that can never match
+        st.block[1:] = cfg.mask_token_id
+
+    out, Ls, _ = O.generate(cfg, w, prompt, sh.k, N_NEW, draft_hook=hook)
+    assert out == ar_tokens[:N_NEW]
+    assert set(Ls) == {1}
+
+
+def test_tidar_equals_ar_perfect_and_partial_drafts(model, ar_tokens):
+    sh, cfg, w, prompt = model
+    k = sh.k
+    n0 = len(prompt)
+
+    def perfect(st):
+        e = st.n - n0                  # tokens emitted before block[0]
+        st.block[1:] = ar_tokens[e + 1:e + k]
+
+    out, Ls, _ = O.generate(cfg, w, prompt, k, N_NEW, draft_hook=perfect)
+    assert out == ar_tokens[:N_NEW]
+    assert set(Ls) == {k}
+
+    def two_right(st):
+        e = st.n - n0
+        st.block[1:] = ar_tokens[e + 1:e + k]
+        st.block[3] = (st.block[3] + 1) % (sh.vocab - 1)
+
+    out, Ls, _ = O.generate(cfg, w, prompt, k, N_NEW, draft_hook=two_right)
+    assert out == ar_tokens[:N_NEW]
+    assert set(Ls) == {3}
+
+
+# ---------------------------------------------------------------- causal section is plain AR
+def test_causal_slots_equal_plain_causal_forward(model):
+    sh, cfg, w, prompt = model
+    st, _ = O.prefill(cfg, w, prompt, sh.k)
+    st.block[1:] = [11, 22, 33]
+    seq = list(prompt) + [int(t) for t in st.block]
+    so = O.step(cfg, w, st)
+    ref = O.causal_forward(cfg, w, seq)
+    n = len(prompt)
+    np.testing.assert_allclose(so.fwd.logits[:sh.k], ref.logits[n:n + sh.k], rtol=1e-9, atol=1e-11)
+    for l in range(cfg.n_layers):
+        np.testing.assert_allclose(so.fwd.k_new[l][:sh.k], ref.k_new[l][n:n + sh.k], rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------- exact KV cache
+def test_kv_cache_equals_one_causal_pass(model):
+    sh, cfg, w, prompt = model
+    out, Ls, st = O.generate(cfg, w, prompt, sh.k, N_NEW)
+    assert st.n == len(prompt) + sum(Ls)
+    ref = O.causal_forward(cfg, w, st.tokens[:st.n])
+    for l in range(cfg.n_layers):
+        assert st.k_cache[l].shape == (st.n, cfg.n_kv_heads, cfg.head_dim)
+        np.testing.assert_allclose(st.k_cache[l], ref.k_new[l], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(st.v_cache[l], ref.v_new[l], rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------- pre-drafts
+@pytest.mark.parametrize("forced", [1, 2, 4])
+def test_selected_predraft_equals_fresh_first_pass(model, forced):
+    sh, cfg, w, prompt = model
+    st, _ = O.prefill(cfg, w, prompt, sh.k)
+    so = O.step(cfg, w, st, forced=forced)
+    # a first pass over everything committed so far drafts from the same context
+    st2, c2, fo2 = O.prefill(cfg, w, st.tokens[:st.n], sh.k, return_forward=True)
+    assert c2 == st.block[0]
+    np.testing.assert_array_equal(st2.block, st.block)
+    g_step = so.fwd.logits[sh.k + (forced - 1) * sh.k: sh.k + forced * sh.k]
+    np.testing.assert_allclose(g_step, fo2.logits[st.n:], rtol=1e-9, atol=1e-11)
+
+
+def test_first_mask_slot_and_ar_row_predict_the_same_position(model):
+    # Section 4.4.3: with beta = 0 the verified token comes from the first slot of
+    # the block; the positions line up, so the layout's position ids must agree.
+    sh, cfg, w, prompt = model
+    _, _, _, pos = O.slot_layout(len(prompt), sh.k)
+    for b in range(sh.k):
+        assert pos[sh.k + b * sh.k] == pos[b] + 1
+
+
+def test_beta_mixes_logits_for_verification(model):
+    sh, cfg, w, prompt = model
+    for beta in (1.0, 0.5, 0.0):
+        cfg_b = replace(cfg, beta=beta)
+        st, _ = O.prefill(cfg_b, w, prompt, sh.k)
+        so = O.step(cfg_b, w, st)
+        a = so.fwd.logits[:sh.k]
+        g0 = so.fwd.logits[sh.k:].reshape(sh.k, sh.k, -1)[:, 0]
+        np.testing.assert_array_equal(so.targets, np.argmax(beta * a + (1 - beta) * g0, axis=-1))
+
+
+# ---------------------------------------------------------------- planted mistakes must be caught
+def _with_mask(monkeypatch, fn):
+    orig = O.build_decode_mask
+
+    def patched(n, k):
+        m = orig(n, k).copy()
+        fn(m, n, k)
+        return m
+
+    monkeypatch.setattr(O, "build_decode_mask", patched)
+
+
+def test_planted_causal_sees_mask_slot_breaks_ar_equivalence(model, ar_tokens, monkeypatch):
+    sh, cfg, w, prompt = model
+    _with_mask(monkeypatch, lambda m, n, k: m.__setitem__((slice(0, k), slice(n + k, n + 2 * k)), True))
+    st, _ = O.prefill(cfg, w, prompt, sh.k)
+    seq = list(prompt) + [int(t) for t in st.block]
+    so = O.step(cfg, w, st)
+    ref = O.causal_forward(cfg, w, seq)
+    assert np.abs(so.fwd.logits[:sh.k] - ref.logits[len(prompt):len(prompt) + sh.k]).max() > 1e-6
+
+
+def test_planted_block_sees_one_more_draft_breaks_predraft_pin(model, monkeypatch):
+    sh, cfg, w, prompt = model
+
+    def widen(m, n, k):               # block b also sees causal slot b+1
+        for b in range(k - 1):
+            m[k + b * k:k + (b + 1) * k, n + b + 1] = True
+
+    _with_mask(monkeypatch, widen)
+    st, _ = O.prefill(cfg, w, prompt, sh.k)
+    st.block[1:] = [11, 22, 33]
+    so = O.step(cfg, w, st, forced=2)
+    monkeypatch.undo()
+    _, _, fo2 = O.prefill(cfg, w, st.tokens[:st.n], sh.k, return_forward=True)
+    g_step = so.fwd.logits[sh.k + sh.k: sh.k + 2 * sh.k]
+    assert np.abs(g_step - fo2.logits[st.n:]).max() > 1e-6
+
+
+def test_planted_wrong_mask_position_breaks_predraft_pin(model, monkeypatch):
+    sh, cfg, w, prompt = model
+    orig = O.slot_layout
+
+    def shifted(n, k):
+        kind, blk, idx, pos = orig(n, k)
+        pos = pos.copy()
+        pos[k:] -= 1                  # label-shifted positions: the reading the paper rules out
+        return kind, blk, idx, pos
+
+    monkeypatch.setattr(O, "slot_layout", shifted)
+    st, _ = O.prefill(cfg, w, prompt, sh.k)
+    so = O.step(cfg, w, st, forced=1)
+    monkeypatch.undo()
+    _, _, fo2 = O.prefill(cfg, w, st.tokens[:st.n], sh.k, return_forward=True)
+    assert np.abs(so.fwd.logits[sh.k:2 * sh.k] - fo2.logits[st.n:]).max() > 1e-6
