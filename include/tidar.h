@@ -1,0 +1,186 @@
+/*
+ * tidar.h - C ABI of the TiDAR single-forward decode step for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the decode path of "TiDAR: Think in Diffusion, Talk in
+ * Autoregression" on one GPU: a first pass over the prompt (tidar_prefill) and
+ * then identical-shape decode steps (tidar_step).  Each step is ONE transformer
+ * forward over k*(k+1) token slots per sequence (paper, Section 3.3 footnote):
+ * the k tokens proposed by the previous step, encoded causally against the
+ * exact KV cache, plus k blocks of k mask tokens that pre-draft the next block
+ * for every possible acceptance outcome (paper, Section 1 "three sections",
+ * Section 3.2, figure "TiDAR Architecture").  After the forward the step keeps
+ * the longest prefix of drafts that agree with the autoregressive prediction,
+ * picks the pre-draft that matches that outcome and commits only the accepted
+ * tokens' KV (Section 3.2; Section 3.3 "evict the KV cache").
+ *
+ * Conventions
+ *   - Every entry point returns TIDAR_OK (0) or a negative TIDAR_E* code and
+ *     leaves the context unchanged on error.  Nothing throws, aborts or traps.
+ *     tidar_last_error() gives a human-readable message for the last failure.
+ *   - "host" / "device" on a pointer says where the memory lives.
+ *   - Weights and the arena are BORROWED: the caller allocates them (for
+ *     instance through PyTorch), keeps them alive until tidar_free and must
+ *     not touch the arena while the context exists.
+ *   - All work is enqueued on the CUDA stream given to tidar_init.  tidar_prefill
+ *     and tidar_step synchronise that stream before they return the tokens.
+ *   - There is no CPU fallback: without a CUDA device tidar_init fails.
+ */
+#ifndef TIDAR_H_
+#define TIDAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TIDAR_OK               0
+#define TIDAR_EINVAL          -1   /* bad argument or unsupported shape                 */
+#define TIDAR_ECAPACITY       -2   /* sequence would outgrow max_seq_len / the KV pool   */
+#define TIDAR_ENOMEM          -3   /* arena too small                                    */
+#define TIDAR_ECUDA           -4   /* a CUDA call failed (message has the CUDA error)    */
+#define TIDAR_EDEVICE_TIMEOUT -5   /* a bounded device-side wait gave up                 */
+
+typedef struct tidar_ctx tidar_ctx;             /* opaque; owned by the library */
+
+/* Model and capacity description; plain data, copied by tidar_init. */
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t tie_lm_head;      /* informational: 1 if weights.lm_head == weights.embed        */
+  float   rms_eps;          /* RMSNorm epsilon                                             */
+  float   rope_theta;       /* RoPE base; rotate-half pairing (i, i + head_dim/2)          */
+  int32_t mask_token_id;    /* id fed to every diffusion (mask) slot                       */
+  int32_t k_max;            /* largest draft block length; k is chosen per prefill         */
+  int32_t max_batch;        /* sequences a context can hold and step together              */
+  int32_t max_seq_len;      /* per sequence; a step needs n + 2k <= max_seq_len            */
+  int32_t page_size;        /* KV page length in tokens (64)                               */
+  float   beta;             /* verification mix (Section 4.4.3); only 1.0 is implemented   */
+  float   temperature;      /* 0 = greedy; only greedy is implemented                      */
+  uint64_t sample_seed;     /* reserved for seeded sampling                                */
+  int32_t debug;            /* bit 0: keep per-layer hidden states and full logits of the
+                               last pass for the tidar_debug_get_* calls (costs memory:
+                               rows*vocab*4 bytes); bit 1: overwrite evicted KV slots with
+                               NaN after each step (proves nothing reads them)             */
+  int32_t impl;             /* 0: tensor-core kernels (tcgen05/TMEM/TMA);
+                               1: plain fp32-accumulate CUDA-core kernels ("replay"), a
+                               slow diagnostic path with the same data flow               */
+} tidar_config;
+
+/* BORROWED device pointers.  Matrices are bf16, row-major [out_features][in_features].
+ *   wqkv[l]      : [(n_q_heads + 2*n_kv_heads)*head_dim][d_model], rows = Q heads, K heads, V heads
+ *   wo[l]        : [d_model][n_q_heads*head_dim]
+ *   w_gate_up[l] : [2*d_ffn][d_model], row 2f = gate row f, row 2f+1 = up row f (interleaved so
+ *                  that one tile of output rows holds matching gate/up pairs)
+ *   w_down[l]    : [d_model][d_ffn]
+ *   embed, lm_head : [vocab][d_model];  *_norm : [d_model] bf16 gains
+ * The six per-layer arrays are HOST arrays of n_layers device pointers.            */
+typedef struct {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *attn_norm, *const *wqkv, *const *wo;
+  const void *const *ffn_norm, *const *w_gate_up, *const *w_down;
+} tidar_weights;
+
+/* Bytes of device memory the context needs for cfg (KV pages, activations, scratch).
+ * The caller allocates that much (256-byte aligned) and passes it to tidar_init.  */
+int tidar_arena_bytes(const tidar_config *cfg, size_t *out_bytes);
+
+/* Validate cfg, adopt the weights and the arena, build TMA descriptors, create the
+ * context.  cuda_stream is a cudaStream_t (NULL = default stream).
+ * Errors: EINVAL (shape not supported: head_dim must be 64 or 128, d_model and d_ffn
+ * multiples of 64, page_size 64, ...), ENOMEM (arena_bytes too small), ECUDA.      */
+int tidar_init(const tidar_config *cfg, const tidar_weights *weights,
+               void *arena /*device*/, size_t arena_bytes, void *cuda_stream, tidar_ctx **out);
+
+/* First pass for sequence slot `seq` (0 <= seq < max_batch), replacing whatever the
+ * slot held (paper, Section 3.2 "In the start of the generation"; Appendix B): the
+ * prompt is encoded causally and its KV cached; one block of k mask tokens is
+ * appended with bidirectional attention.  Emits the first settled token (argmax of
+ * the last prompt row) to *out_first_token and stores the first draft block.
+ * Needs 1 <= n_prompt, 1 <= k <= k_max, n_prompt + 2k <= max_seq_len.             */
+int tidar_prefill(tidar_ctx *ctx, int32_t seq, const int32_t *prompt_ids /*host*/, int32_t n_prompt,
+                  int32_t k, int32_t *out_first_token /*host*/);
+
+/* One decode step for the listed sequences (all prefetched with the same k).
+ * forced_accept: NULL, or per sequence 0 = natural acceptance, L in [1,k] = accept
+ * exactly L slots whatever the drafts were (benchmark hook; not in the paper).
+ * On return out_n[i] = L_i and out_tokens[i*k_max .. i*k_max+L_i) = the L_i new tokens:
+ * the accepted drafts followed by the freshly verified token.  The committed KV
+ * length of sequence i grows by L_i; rejected slots are evicted.
+ * Errors: EINVAL, ECAPACITY (n + 2k > max_seq_len, checked before any launch).     */
+int tidar_step(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs,
+               const int32_t *forced_accept /*host,[n_seqs] or NULL*/,
+               int32_t *out_tokens /*host,[n_seqs][k_max]*/, int32_t *out_n /*host,[n_seqs]*/);
+
+/* Same as tidar_step but returns after enqueueing; results are fetched (and the
+ * stream synchronised) by tidar_step_wait.  Used to time steps back to back.
+ * Forced acceptance lengths are required (the host must know every sequence's
+ * length to check capacity without reading the device).                           */
+int tidar_step_async(tidar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, const int32_t *forced_accept);
+int tidar_step_wait(tidar_ctx *ctx, int32_t *out_tokens /*host,[n_seqs][k_max]*/, int32_t *out_n /*host*/);
+
+/* Release the context (host state only; arena and weights belong to the caller). */
+int tidar_free(tidar_ctx *ctx);
+
+/* Message for the most recent error on ctx (or for the last failed tidar_init when
+ * ctx is NULL).  The pointer stays valid until the next call on the same ctx.     */
+const char *tidar_last_error(const tidar_ctx *ctx);
+
+/* Committed KV length n of a sequence slot (host bookkeeping), or a negative code. */
+int tidar_seq_len(const tidar_ctx *ctx, int32_t seq);
+
+/* Number of kernels the library launched since tidar_init (for launch accounting). */
+int64_t tidar_launch_count(const tidar_ctx *ctx);
+
+/* ---- rewind / teacher forcing (parity tests) ------------------------------------ */
+/* Overwrite the next step's causal section of a sequence: block[0] is the settled
+ * token at position n, block[1..k) the drafts.                                      */
+int tidar_debug_set_block(tidar_ctx *ctx, int32_t seq, const int32_t *block /*host,[k]*/);
+int tidar_debug_get_block(tidar_ctx *ctx, int32_t seq, int32_t *block /*host,[k]*/);
+/* Results of the last pass; need cfg.debug bit 0.  Row r of a decode step is slot
+ * r % (k*(k+1)) of the (r / (k*(k+1)))-th listed sequence; for a prefill the rows are
+ * the last chunk's rows (see tidar_debug_last_rows).                               */
+int tidar_debug_last_rows(const tidar_ctx *ctx, int32_t *n_rows, int32_t *first_row_position);
+int tidar_debug_get_logits(tidar_ctx *ctx, int32_t row0, int32_t n_rows, float *out /*host,[n_rows][vocab]*/);
+/* layer in [0, n_layers]: input of that layer; n_layers = input of the final norm. */
+int tidar_debug_get_hidden(tidar_ctx *ctx, int32_t layer, int32_t row0, int32_t n_rows,
+                           float *out /*host,[n_rows][d_model]*/);
+int tidar_debug_get_argmax(tidar_ctx *ctx, int32_t row0, int32_t n_rows, int32_t *out /*host*/);
+/* Cached K and V (bf16 bit patterns) of positions [pos0, pos0+npos) in canonical
+ * [npos][n_kv_heads][head_dim] order, gathered from the pages.                     */
+int tidar_debug_get_kv(tidar_ctx *ctx, int32_t seq, int32_t layer, int32_t pos0, int32_t npos,
+                       uint16_t *k_out /*host*/, uint16_t *v_out /*host*/);
+/* Per-kernel-class device time (ms) of the last pass, measured with CUDA events when
+ * enabled with tidar_debug_set_timing(ctx, 1).  classes: see TIDAR_TC_* below.     */
+#define TIDAR_TC_EMBED   0
+#define TIDAR_TC_NORM    1
+#define TIDAR_TC_GEMM    2
+#define TIDAR_TC_ROPE    3
+#define TIDAR_TC_ATTN    4
+#define TIDAR_TC_LMHEAD  5
+#define TIDAR_TC_VERIFY  6
+#define TIDAR_TC_COUNT   7
+int tidar_debug_set_timing(tidar_ctx *ctx, int32_t on);
+int tidar_debug_get_timing(tidar_ctx *ctx, float *ms /*host,[TIDAR_TC_COUNT]*/);
+
+/* ---- structured-mask attention alone (microbenchmark and unit parity) -------------
+ * Runs the step's attention kernel on caller-provided tensors (all DEVICE, bf16):
+ *   q        [n_seqs*T][n_q_heads][head_dim], T = k*(k+1), slot order of a decode step
+ *   k_pages, v_pages : page pools [n_pages][n_kv_heads][page_size][head_dim]; the
+ *              cached prefix AND the k causal slots of the step (positions n..n+k-1)
+ *              live there
+ *   page_table [n_seqs][pages_per_seq] int32, seq_len [n_seqs] int32 (= n per sequence)
+ *   k_local, v_local [n_seqs*k*k][n_kv_heads][head_dim] : K/V of the mask slots
+ *   out      [n_seqs*T][n_q_heads*head_dim]
+ * Mask per the decode-step definition: causal slot j sees positions < n+j+1; mask
+ * slot (b,i) sees positions < n+b+1 plus the k local slots of block b.
+ * Uses ctx only for its stream, kernel implementation choice and scratch.          */
+int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const void *v_pages,
+                    const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
+                    const void *k_local, const void *v_local, void *out,
+                    int32_t n_seqs, int32_t k);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* TIDAR_H_ */

@@ -1,0 +1,46 @@
+// Shared declarations for the TiDAR decode-step kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+// Per-row metadata of one pass (a decode step or a prefill chunk).  A "row" is one
+// token slot.  Every row attends to cache positions [0, nvis) of its sequence plus
+// the nloc local (never cached) K/V rows starting at loc0.  This one rule covers the
+// whole structured mask of the decode step: causal slot j has its K/V written to the
+// cache at position n+j before attention, so it sees nvis = n+j+1 and nothing local;
+// mask slot (b,i) sees nvis = n+b+1 (the prefix plus causal slots 0..b) and the k
+// local slots of its own block.
+struct RowMeta {
+  int32_t *ids;        // token id
+  int32_t *pos;        // position id (RoPE)
+  int32_t *seq;        // sequence slot
+  int32_t *nvis;       // visible cache positions
+  int32_t *loc0;       // first local K/V row (or 0 when nloc == 0)
+  int32_t *nloc;       // number of local K/V rows visible
+  int32_t *cache_pos;  // where this row's K/V go in the cache, or -1
+  int32_t *local_idx;  // where this row's K/V go in the local scratch, or -1
+};
+
+struct KvGeom {
+  int32_t n_kv_heads, head_dim, page_size, pages_per_seq;
+  const int32_t *page_table;   // [max_batch][pages_per_seq]
+};
+
+__device__ __forceinline__ size_t kv_row_offset(const KvGeom &g, int seq, int position, int kvh) {
+  int page = g.page_table[(size_t)seq * g.pages_per_seq + position / g.page_size];
+  return (((size_t)page * g.n_kv_heads + kvh) * g.page_size + (position % g.page_size)) * (size_t)g.head_dim;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}

@@ -1,0 +1,302 @@
+// Slot assembly, embedding, RMSNorm, RoPE + KV placement, SwiGLU, argmax,
+// draft/verify and KV commit kernels of the TiDAR decode step.
+#pragma once
+#include "common.cuh"
+
+// ---------------------------------------------------------------------------
+// Slot assembly + embedding gather for a decode step.
+// Slot layout per sequence (k causal slots, then k blocks of k mask slots;
+// paper Section 3.3 footnote, figure "TiDAR Attention Masks"):
+//   causal j       : token block[j], position n+j
+//   mask (b, i)    : [MASK], position n+b+1+i (no label shift: a mask slot predicts
+//                    its own position; paper Section 4.4.3)
+// One block per row; also snapshots n into step_n for the commit kernel.
+// ---------------------------------------------------------------------------
+__global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ seq_len,
+                                     const int32_t *__restrict__ block_ids, int k, int k_max, int mask_id,
+                                     int32_t *__restrict__ step_n, const bf16 *__restrict__ embed, int d,
+                                     float *__restrict__ X) {
+  const int T = k * (k + 1);
+  const int r = blockIdx.x;
+  const int s = r / T, slot = r % T;
+  const int seq = step_seqs[s];
+  const int n = seq_len[seq];
+  int id;
+  if (slot < k) id = block_ids[seq * k_max + slot]; else id = mask_id;
+  if (threadIdx.x == 0) {
+    if (slot == 0) step_n[s] = n;
+    m.seq[r] = seq;
+    m.ids[r] = id;
+    if (slot < k) {
+      m.pos[r] = n + slot; m.nvis[r] = n + slot + 1; m.loc0[r] = 0; m.nloc[r] = 0;
+      m.cache_pos[r] = n + slot; m.local_idx[r] = -1;
+    } else {
+      const int b = (slot - k) / k, i = (slot - k) % k;
+      m.pos[r] = n + b + 1 + i; m.nvis[r] = n + b + 1; m.loc0[r] = s * k * k + b * k; m.nloc[r] = k;
+      m.cache_pos[r] = -1; m.local_idx[r] = s * k * k + b * k + i;
+    }
+  }
+  const bf16 *e = embed + (size_t)id * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) X[(size_t)r * d + c] = __bfloat162float(e[c]);
+}
+
+// Prefill chunk: rows g = row0 .. row0+rows-1 of [prompt ; k mask tokens]
+// (paper Section 3.2, Appendix B): prompt rows causal, mask rows see the whole
+// prompt and each other.
+__global__ void assemble_prefill_kernel(RowMeta m, int seq, int row0, int n_prompt, int k, int mask_id,
+                                        const int32_t *__restrict__ prompt, const bf16 *__restrict__ embed, int d,
+                                        float *__restrict__ X) {
+  const int r = blockIdx.x;
+  const int g = row0 + r;
+  const int id = g < n_prompt ? prompt[g] : mask_id;
+  if (threadIdx.x == 0) {
+    m.seq[r] = seq; m.ids[r] = id; m.pos[r] = g;
+    if (g < n_prompt) {
+      m.nvis[r] = g + 1; m.loc0[r] = 0; m.nloc[r] = 0; m.cache_pos[r] = g; m.local_idx[r] = -1;
+    } else {
+      m.nvis[r] = n_prompt; m.loc0[r] = 0; m.nloc[r] = k; m.cache_pos[r] = -1; m.local_idx[r] = g - n_prompt;
+    }
+  }
+  const bf16 *e = embed + (size_t)id * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) X[(size_t)r * d + c] = __bfloat162float(e[c]);
+}
+
+// Row metadata for the stand-alone attention entry point (same slot layout as a step).
+__global__ void attn_meta_kernel(RowMeta m, const int32_t *__restrict__ seq_len, int k, int R) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  const int T = k * (k + 1);
+  const int s = r / T, slot = r % T;
+  const int n = seq_len[s];
+  m.seq[r] = s;
+  if (slot < k) {
+    m.pos[r] = n + slot; m.nvis[r] = n + slot + 1; m.loc0[r] = 0; m.nloc[r] = 0;
+  } else {
+    const int b = (slot - k) / k;
+    m.pos[r] = n + b + 1 + (slot - k) % k; m.nvis[r] = n + b + 1; m.loc0[r] = s * k * k + b * k; m.nloc[r] = k;
+  }
+}
+
+// cos/sin of pos * theta^(-2i/hd), evaluated in double once per pass (shared by every
+// layer and head), stored as float.
+__global__ void rope_table_kernel(const int32_t *__restrict__ pos, int R, int half, double theta,
+                                  float *__restrict__ cs, float *__restrict__ sn) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= R * half) return;
+  const int r = t / half, i = t % half;
+  const double inv = pow(theta, -(double)i / (double)half);
+  double s, c;
+  sincos((double)pos[r] * inv, &s, &c);
+  cs[t] = (float)c; sn[t] = (float)s;
+}
+
+// ---------------------------------------------------------------------------
+// Residual update + RMSNorm.  X (fp32 residual stream) += sum over the S split-K
+// partial results of the previous projection (fixed order: deterministic), then
+// A = bf16(X * rsqrt(mean(X^2) + eps) * gain).  One block per row.
+// ---------------------------------------------------------------------------
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials, int S, size_t partial_stride,
+                      const bf16 *__restrict__ gain, float eps, int d, bf16 *__restrict__ A) {
+  extern __shared__ float row[];
+  __shared__ float red[THREADS / 32];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d; c += THREADS) {
+    float v = X[(size_t)r * d + c];
+    for (int s = 0; s < S; ++s) v += partials[s * partial_stride + (size_t)r * d + c];
+    row[c] = v;
+    ss += v * v;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < THREADS / 32; ++i) tot += red[i];
+  const float inv = rsqrtf(tot / (float)d + eps);
+  for (int c = threadIdx.x; c < d; c += THREADS) {
+    const float v = row[c];
+    if (S > 0) X[(size_t)r * d + c] = v;
+    A[(size_t)r * d + c] = __float2bfloat16(v * inv * __bfloat162float(gain[c]));
+  }
+}
+
+// ---------------------------------------------------------------------------
+// RoPE + KV placement.  Input: S split-K partials of the QKV projection, fp32
+// [S][R][(Hq+2Hkv)*hd].  Q heads are rotated and stored bf16 [R][Hq][hd]; K heads are
+// rotated, V heads copied; both go to the paged cache at the row's cache position
+// (causal slots: kept if accepted, evicted otherwise; paper Section 3.3) or to the
+// step-local scratch (mask slots, never cached).  Grid (R, Hq+2Hkv), hd/2 threads.
+// ---------------------------------------------------------------------------
+__global__ void rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
+                               RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
+                               bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
+                               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
+  const int r = blockIdx.x, h = blockIdx.y, i = threadIdx.x, half = hd / 2;
+  const int N = (Hq + 2 * Hkv) * hd;
+  const size_t base = (size_t)r * N + (size_t)h * hd;
+  float x1 = 0.f, x2 = 0.f;
+  for (int s = 0; s < S; ++s) {
+    x1 += partials[s * partial_stride + base + i];
+    x2 += partials[s * partial_stride + base + i + half];
+  }
+  bf16 *dst;
+  if (h < Hq) {
+    dst = Q + ((size_t)r * Hq + h) * hd;
+  } else {
+    const bool isk = h < Hq + Hkv;
+    const int kvh = isk ? h - Hq : h - Hq - Hkv;
+    const int cp = m.cache_pos[r];
+    if (cp >= 0) dst = (isk ? Kpool : Vpool) + kv_row_offset(g, m.seq[r], cp, kvh);
+    else dst = (isk ? Kloc : Vloc) + ((size_t)m.local_idx[r] * Hkv + kvh) * hd;
+    if (!isk) {  // V: no rotation
+      dst[i] = __float2bfloat16(x1); dst[i + half] = __float2bfloat16(x2);
+      return;
+    }
+  }
+  const float c = cs[r * half + i], s = sn[r * half + i];
+  dst[i] = __float2bfloat16(x1 * c - x2 * s);
+  dst[i + half] = __float2bfloat16(x2 * c + x1 * s);
+}
+
+// SwiGLU on an fp32 [R][2*ffn] projection whose columns interleave (gate_f, up_f).
+__global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16 *__restrict__ H) {
+  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (size_t)R * ffn) return;
+  const float g = GU[2 * t], u = GU[2 * t + 1];
+  H[t] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+}
+
+// Running per-row argmax over a chunk of logits [R][ncols] (fp32, leading dim ld)
+// that covers vocabulary ids [col0, col0+ncols).  Lowest index wins ties; NaN never
+// wins.  Optionally copies the chunk into a full [R][vocab] dump.
+__global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int ncols, int col0, int first,
+                                    float *__restrict__ best_val, int32_t *__restrict__ best_idx,
+                                    float *__restrict__ dump, int vocab) {
+  const int r = blockIdx.x;
+  float bv = -INFINITY; int bi = 0x7fffffff;
+  for (int c = threadIdx.x; c < ncols; c += blockDim.x) {
+    const float v = L[(size_t)r * ld + c];
+    if (dump) dump[(size_t)r * vocab + col0 + c] = v;
+    if (v > bv) { bv = v; bi = col0 + c; }
+  }
+  __shared__ float sv[32]; __shared__ int si[32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o); const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+      if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
+    if (!first) {
+      const float pv = best_val[r]; const int pi = best_idx[r];
+      if (pv > bv || (pv == bv && pi < bi) || bi == 0x7fffffff) { bv = pv; bi = pi; }
+    }
+    if (bi == 0x7fffffff) bi = 0;
+    best_val[r] = bv; best_idx[r] = bi;
+  }
+}
+
+// Final argmax over per-CTA partial results [G][R] produced by the fused LM-head
+// epilogue: one thread per row scans the G candidates in order.
+__global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t *__restrict__ pi, int G, int R,
+                                    float *__restrict__ best_val, int32_t *__restrict__ best_idx) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  float bv = -INFINITY; int bi = 0x7fffffff;
+  for (int g = 0; g < G; ++g) {
+    const float v = pv[(size_t)g * R + r]; const int i = pi[(size_t)g * R + r];
+    if (i >= 0 && (v > bv || (v == bv && i < bi))) { bv = v; bi = i; }
+  }
+  if (bi == 0x7fffffff) bi = 0;
+  best_val[r] = bv; best_idx[r] = bi;
+}
+
+// ---------------------------------------------------------------------------
+// Draft / verify / select (paper Section 3.2; Section 4.4.3 with beta = 1).
+// One warp per sequence, lane i = causal slot i:
+//   target_i = argmax of causal slot i's logits (prediction for position n+i+1);
+//   draft i >= 1 agrees iff block[i] == target_{i-1};
+//   L = 1 + length of the leading run of agreeing drafts (slot 0 is settled), or the
+//   forced value;  emitted = block[1..L-1], target_{L-1};
+//   next block = target_{L-1}, then the argmax of mask slots (L-1, 1..k-1).
+// ---------------------------------------------------------------------------
+__global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const int32_t *__restrict__ step_seqs,
+                                     const int32_t *__restrict__ forced, int k, int k_max,
+                                     int32_t *__restrict__ block_ids, int32_t *__restrict__ step_L,
+                                     int32_t *__restrict__ out /*[n_seqs][k_max+1]*/) {
+  const int s = blockIdx.x, lane = threadIdx.x;
+  const int T = k * (k + 1);
+  const int seq = step_seqs[s];
+  const int32_t *ids = arg_ids + (size_t)s * T;
+  int32_t *blk = block_ids + (size_t)seq * k_max;
+  const int tgt = lane < k ? ids[lane] : -1;
+  const int mine = lane < k ? blk[lane] : -2;
+  const int prev_tgt = __shfl_up_sync(0xffffffffu, tgt, 1);
+  const bool agree = lane == 0 || (lane < k && mine == prev_tgt);
+  const unsigned bits = __ballot_sync(0xffffffffu, agree);
+  int L = __ffs(~bits) - 1;            // leading run of ones; bit 0 is always set
+  if (L > k || L < 0) L = k;           // all 32 lanes agreeing gives ffs(0) = 0
+  const int f = forced ? forced[s] : 0;
+  if (f > 0) L = f;
+  const int t_last = __shfl_sync(0xffffffffu, tgt, L - 1);
+  const int next_draft = (lane >= 1 && lane < k) ? ids[k + (L - 1) * k + lane] : 0;
+  const int shifted = __shfl_down_sync(0xffffffffu, mine, 1);     // block[lane+1]
+  __syncwarp();
+  if (lane < k) {
+    out[(size_t)s * (k_max + 1) + 1 + lane] = lane < L - 1 ? shifted : (lane == L - 1 ? t_last : -1);
+    blk[lane] = lane == 0 ? t_last : next_draft;
+  }
+  if (lane == 0) { out[(size_t)s * (k_max + 1)] = L; step_L[s] = L; }
+}
+
+// First-pass finish: settled token = argmax of the last prompt row; drafts = argmax
+// of mask rows 1..k-1 (paper Section 3.2, start of generation).
+__global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int row_last_prompt, int k, int k_max, int seq,
+                                      int n_prompt, int32_t *__restrict__ block_ids, int32_t *__restrict__ seq_len,
+                                      int32_t *__restrict__ out) {
+  const int i = threadIdx.x;
+  if (i < k) block_ids[(size_t)seq * k_max + i] = i == 0 ? arg_ids[row_last_prompt] : arg_ids[row_last_prompt + 1 + i];
+  if (i == 0) { seq_len[seq] = n_prompt; out[0] = arg_ids[row_last_prompt]; }
+}
+
+// ---------------------------------------------------------------------------
+// KV commit / evict (paper Section 3.3): the k causal slots' K/V were written to
+// the cache at positions n..n+k-1 during the pass; committing L of them is
+// n <- n + L, after which positions n+L..n+k-1 are dead and get overwritten by the
+// next step.  With poison != 0 the dead slots are filled with NaN in every layer, so
+// any later read of evicted data would surface.  Grid (n_seqs, n_layers).
+// ---------------------------------------------------------------------------
+__global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ step_n,
+                                 const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, int poison,
+                                 KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride) {
+  const int s = blockIdx.x, l = blockIdx.y;
+  const int seq = step_seqs[s];
+  const int n = step_n[s], L = step_L[s];
+  if (l == 0 && threadIdx.x == 0) seq_len[seq] = n + L;
+  if (!poison) return;
+  bf16 *Kp = kv_base + (size_t)(2 * l) * pool_stride, *Vp = Kp + pool_stride;
+  const int per = g.n_kv_heads * g.head_dim;
+  const bf16 nanv = __ushort_as_bfloat16((unsigned short)0x7fc0);
+  for (int t = threadIdx.x; t < (k - L) * per; t += blockDim.x) {
+    const int p = n + L + t / per, kvh = (t % per) / g.head_dim, c = t % g.head_dim;
+    const size_t off = kv_row_offset(g, seq, p, kvh) + c;
+    Kp[off] = nanv; Vp[off] = nanv;
+  }
+}
+
+// Gather cached K/V rows into canonical [npos][Hkv][hd] order (debug read-back).
+__global__ void kv_gather_kernel(const bf16 *__restrict__ Kp, const bf16 *__restrict__ Vp, KvGeom g, int seq, int pos0,
+                                 bf16 *__restrict__ ko, bf16 *__restrict__ vo) {
+  const int p = blockIdx.x, kvh = blockIdx.y;
+  const size_t off = kv_row_offset(g, seq, pos0 + p, kvh);
+  for (int c = threadIdx.x; c < g.head_dim; c += blockDim.x) {
+    ko[((size_t)p * g.n_kv_heads + kvh) * g.head_dim + c] = Kp[off + c];
+    vo[((size_t)p * g.n_kv_heads + kvh) * g.head_dim + c] = Vp[off + c];
+  }
+}

@@ -1,0 +1,582 @@
+// C-ABI entry points and per-step orchestration of the TiDAR decode path.
+#include "../../include/tidar.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels_basic.cuh"
+#include "kernels_replay.cuh"
+
+namespace {
+
+std::string g_init_error;
+
+struct SeqState {
+  int n = 0;            // committed KV length
+  int k = 0;            // draft block length chosen at prefill
+  bool active = false;
+  std::vector<int> pages;
+};
+
+struct TimedLaunch { int cls; cudaEvent_t a, b; };
+
+}  // namespace
+
+struct tidar_ctx {
+  tidar_config cfg;
+  cudaStream_t stream = nullptr;
+  // borrowed weights
+  const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  std::vector<const bf16 *> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
+  // geometry
+  int R_cap = 0, T_max = 0, pages_per_seq = 0, n_pages = 0, n_qkv = 0, S_max = 4, lm_chunk = 0;
+  size_t pool_stride = 0;    // elements in one layer's K (or V) pool
+  size_t partial_stride = 0; // elements between split-K partial slabs
+  // arena carve-out (device)
+  bf16 *kv = nullptr;
+  RowMeta meta{};
+  int32_t *d_seq_len = nullptr, *d_block = nullptr, *d_page_table = nullptr, *d_step_seqs = nullptr, *d_forced = nullptr,
+          *d_step_n = nullptr, *d_step_L = nullptr, *d_out = nullptr, *d_prompt = nullptr, *d_arg_idx = nullptr;
+  float *X = nullptr, *partials = nullptr, *rope_cos = nullptr, *rope_sin = nullptr, *d_arg_val = nullptr,
+        *dbg_hidden = nullptr, *dbg_logits = nullptr;
+  bf16 *A = nullptr, *Q = nullptr, *Kloc = nullptr, *Vloc = nullptr, *O = nullptr, *H = nullptr, *dbg_kv = nullptr;
+  // host state
+  std::vector<SeqState> seqs;
+  std::vector<int> free_pages;
+  int32_t *h_pinned = nullptr;     // [max_batch*(k_max+1)] results + staging
+  int32_t *h_stage = nullptr;      // [2*max_batch] seq list + forced, pinned
+  std::string err;
+  int64_t launches = 0;
+  // last pass
+  int last_rows = 0, last_first_pos = 0;
+  std::vector<int> pending_seqs; std::vector<int> pending_forced; bool pending = false;
+  // timing
+  bool timing = false; std::vector<TimedLaunch> timed; float class_ms[TIDAR_TC_COUNT] = {};
+  int cur_class = 0;
+};
+
+namespace {
+
+int fail(tidar_ctx *c, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap; va_start(ap, fmt); vsnprintf(buf, sizeof buf, fmt, ap); va_end(ap);
+  if (c) c->err = buf; else g_init_error = buf;
+  return code;
+}
+
+#define CUDA_TRY(c, call)                                                                     \
+  do {                                                                                        \
+    cudaError_t e_ = (call);                                                                  \
+    if (e_ != cudaSuccess) return fail((c), TIDAR_ECUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Lays the arena out; with base == nullptr only measures.
+struct Carver {
+  char *base; size_t off = 0;
+  explicit Carver(void *b) : base((char *)b) {}
+  template <typename T> T *take(size_t n) {
+    off = align_up(off, 256);
+    T *p = base ? (T *)(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+int validate(const tidar_config &c, std::string &why) {
+  auto bad = [&](const char *m) { why = m; return TIDAR_EINVAL; };
+  if (c.n_layers < 1 || c.d_model < 64 || c.vocab < 2 || c.d_ffn < 64) return bad("n_layers, d_model, d_ffn, vocab must be positive");
+  if (c.head_dim != 64 && c.head_dim != 128) return bad("head_dim must be 64 or 128");
+  if (c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads) return bad("n_q_heads must be a multiple of n_kv_heads");
+  if (c.d_model % 64 || c.d_ffn % 64) return bad("d_model and d_ffn must be multiples of 64");
+  if (c.page_size != 64) return bad("page_size must be 64");
+  if (c.k_max < 1 || c.k_max > 32) return bad("k_max must be in [1, 32]");
+  if (c.max_batch < 1 || c.max_seq_len < 2 * c.k_max + 1) return bad("max_batch >= 1 and max_seq_len > 2*k_max required");
+  if (c.mask_token_id < 0 || c.mask_token_id >= c.vocab) return bad("mask_token_id out of range");
+  if (c.beta != 1.0f) return bad("only beta = 1 is implemented");
+  if (c.temperature != 0.0f) return bad("only greedy decoding (temperature 0) is implemented");
+  if (c.impl != 1) return bad("impl must be 1 (replay kernels); the tensor-core path is not built into this library yet");
+  if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return bad("rms_eps > 0 and rope_theta > 1 required");
+  return TIDAR_OK;
+}
+
+void layout(tidar_ctx &x, void *arena, size_t *bytes) {
+  const tidar_config &c = x.cfg;
+  x.T_max = c.k_max * (c.k_max + 1);
+  x.R_cap = (int)align_up((size_t)std::max(c.max_batch * x.T_max, 256), 16);
+  x.pages_per_seq = (c.max_seq_len + c.page_size - 1) / c.page_size;
+  x.n_pages = x.pages_per_seq * c.max_batch;
+  x.n_qkv = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  x.pool_stride = (size_t)x.n_pages * c.n_kv_heads * c.page_size * c.head_dim;
+  x.lm_chunk = std::min(c.vocab, 16384);
+  const size_t R = x.R_cap;
+  const size_t widest = std::max<size_t>({(size_t)x.S_max * x.n_qkv, (size_t)x.S_max * c.d_model, (size_t)2 * c.d_ffn,
+                                          (size_t)x.lm_chunk});
+  x.partial_stride = 0;  // set per projection
+  Carver cv(arena);
+  x.kv = cv.take<bf16>((size_t)c.n_layers * 2 * x.pool_stride);
+  x.meta.ids = cv.take<int32_t>(R); x.meta.pos = cv.take<int32_t>(R); x.meta.seq = cv.take<int32_t>(R);
+  x.meta.nvis = cv.take<int32_t>(R); x.meta.loc0 = cv.take<int32_t>(R); x.meta.nloc = cv.take<int32_t>(R);
+  x.meta.cache_pos = cv.take<int32_t>(R); x.meta.local_idx = cv.take<int32_t>(R);
+  x.d_seq_len = cv.take<int32_t>(c.max_batch);
+  x.d_block = cv.take<int32_t>((size_t)c.max_batch * c.k_max);
+  x.d_page_table = cv.take<int32_t>((size_t)c.max_batch * x.pages_per_seq);
+  x.d_step_seqs = cv.take<int32_t>(c.max_batch); x.d_forced = cv.take<int32_t>(c.max_batch);
+  x.d_step_n = cv.take<int32_t>(c.max_batch); x.d_step_L = cv.take<int32_t>(c.max_batch);
+  x.d_out = cv.take<int32_t>((size_t)c.max_batch * (c.k_max + 1));
+  x.d_prompt = cv.take<int32_t>(c.max_seq_len);
+  x.d_arg_idx = cv.take<int32_t>(R); x.d_arg_val = cv.take<float>(R);
+  x.X = cv.take<float>(R * c.d_model);
+  x.partials = cv.take<float>(R * widest);
+  x.rope_cos = cv.take<float>(R * (c.head_dim / 2)); x.rope_sin = cv.take<float>(R * (c.head_dim / 2));
+  x.A = cv.take<bf16>(R * c.d_model);
+  x.Q = cv.take<bf16>(R * c.n_q_heads * c.head_dim);
+  x.O = cv.take<bf16>(R * c.n_q_heads * c.head_dim);
+  const size_t nloc = (size_t)std::max(c.max_batch * c.k_max * c.k_max, c.k_max);
+  x.Kloc = cv.take<bf16>(nloc * c.n_kv_heads * c.head_dim);
+  x.Vloc = cv.take<bf16>(nloc * c.n_kv_heads * c.head_dim);
+  x.H = cv.take<bf16>(R * c.d_ffn);
+  x.dbg_kv = cv.take<bf16>((size_t)2 * 256 * c.n_kv_heads * c.head_dim);
+  if (c.debug & 1) {
+    x.dbg_hidden = cv.take<float>((size_t)(c.n_layers + 1) * R * c.d_model);
+    x.dbg_logits = cv.take<float>(R * (size_t)c.vocab);
+  }
+  *bytes = align_up(cv.off, 256);
+}
+
+// ---- launch bookkeeping -----------------------------------------------------
+struct Launch {
+  tidar_ctx *c; int cls; cudaEvent_t a = nullptr, b = nullptr;
+  Launch(tidar_ctx *c_, int cls_) : c(c_), cls(cls_) {
+    c->launches++;
+    if (c->timing) { cudaEventCreate(&a); cudaEventCreate(&b); cudaEventRecord(a, c->stream); }
+  }
+  ~Launch() {
+    if (c->timing) { cudaEventRecord(b, c->stream); c->timed.push_back({cls, a, b}); }
+  }
+};
+
+void collect_timing(tidar_ctx *c) {
+  for (int i = 0; i < TIDAR_TC_COUNT; ++i) c->class_ms[i] = 0.f;
+  for (auto &t : c->timed) {
+    float ms = 0.f; cudaEventElapsedTime(&ms, t.a, t.b);
+    c->class_ms[t.cls] += ms;
+    cudaEventDestroy(t.a); cudaEventDestroy(t.b);
+  }
+  c->timed.clear();
+}
+
+KvGeom geom(const tidar_ctx *c) {
+  return KvGeom{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, c->pages_per_seq, c->d_page_table};
+}
+
+// ---- projections --------------------------------------------------------------
+// out = A[R][K] * W[N][K]^T as S split-K partial slabs of fp32 [R][N] (replay: S = 1).
+void gemm_partials(tidar_ctx *c, const bf16 *A, const bf16 *W, int R, int N, int K, float *out, int *S_out,
+                   size_t *stride_out, int cls) {
+  Launch l(c, cls);
+  dim3 grid((N + 63) / 64, (R + 63) / 64);
+  gemm_replay_kernel<<<grid, 256, 0, c->stream>>>(A, K, W, K, out, N, R, N, K);
+  *S_out = 1; *stride_out = (size_t)R * N;
+}
+
+void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *Vp, const KvGeom &g, const bf16 *Kl,
+                      const bf16 *Vl, bf16 *O, int R) {
+  Launch l(c, TIDAR_TC_ATTN);
+  const float scale = 1.0f / sqrtf((float)c->cfg.head_dim);
+  dim3 grid(R, c->cfg.n_q_heads);
+  if (c->cfg.head_dim == 128)
+    attn_replay_kernel<128><<<grid, 32, 0, c->stream>>>(Q, Kp, Vp, g, c->meta, Kl, Vl, O, c->cfg.n_q_heads, scale);
+  else
+    attn_replay_kernel<64><<<grid, 32, 0, c->stream>>>(Q, Kp, Vp, g, c->meta, Kl, Vl, O, c->cfg.n_q_heads, scale);
+}
+
+void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t stride, const bf16 *gain) {
+  Launch l(c, TIDAR_TC_NORM);
+  const int d = c->cfg.d_model;
+  rmsnorm_reduce_kernel<256><<<R, 256, d * sizeof(float), c->stream>>>(c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+}
+
+// The transformer stack over R assembled rows (metadata and X already filled).
+// with_head: run final norm + LM head + per-row argmax.
+int forward_rows(tidar_ctx *c, int R, bool with_head) {
+  const tidar_config &cf = c->cfg;
+  const int d = cf.d_model, hd = cf.head_dim, Hq = cf.n_q_heads, Hkv = cf.n_kv_heads;
+  const KvGeom g = geom(c);
+  {
+    Launch l(c, TIDAR_TC_ROPE);
+    const int n = R * (hd / 2);
+    rope_table_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
+  }
+  int S = 0; size_t stride = 0;          // pending partials of the previous down projection
+  for (int l = 0; l < cf.n_layers; ++l) {
+    bf16 *Kp = c->kv + (size_t)(2 * l) * c->pool_stride, *Vp = Kp + c->pool_stride;
+    launch_norm(c, R, c->partials, S, stride, c->attn_norm[l]);
+    if (c->dbg_hidden)
+      CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)l * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, c->stream));
+    gemm_partials(c, c->A, c->wqkv[l], R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    {
+      Launch ll(c, TIDAR_TC_ROPE);
+      rope_kv_kernel<<<dim3(R, Hq + 2 * Hkv), hd / 2, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
+    }
+    launch_attention(c, c->Q, Kp, Vp, g, c->Kloc, c->Vloc, c->O, R);
+    gemm_partials(c, c->O, c->wo[l], R, d, Hq * hd, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    launch_norm(c, R, c->partials, S, stride, c->ffn_norm[l]);
+    gemm_partials(c, c->A, c->wgu[l], R, 2 * cf.d_ffn, d, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    {
+      Launch ll(c, TIDAR_TC_GEMM);
+      const size_t n = (size_t)R * cf.d_ffn;
+      swiglu_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->partials, R, cf.d_ffn, c->H);
+    }
+    gemm_partials(c, c->H, c->wdown[l], R, d, cf.d_ffn, c->partials, &S, &stride, TIDAR_TC_GEMM);
+  }
+  launch_norm(c, R, c->partials, S, stride, c->final_norm);
+  if (c->dbg_hidden)
+    CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)cf.n_layers * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
+                                cudaMemcpyDeviceToDevice, c->stream));
+  if (with_head) {
+    for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
+      const int nc = std::min(c->lm_chunk, cf.vocab - v0);
+      gemm_partials(c, c->A, c->lm_head + (size_t)v0 * d, R, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD);
+      Launch ll(c, TIDAR_TC_LMHEAD);
+      argmax_chunk_kernel<<<R, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab);
+    }
+  }
+  CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
+int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
+  SeqState &s = c->seqs[seq];
+  const int need = (upto_positions + c->cfg.page_size - 1) / c->cfg.page_size;
+  if (need > c->pages_per_seq) return fail(c, TIDAR_ECAPACITY, "sequence %d needs %d pages, limit %d", seq, need, c->pages_per_seq);
+  if ((int)s.pages.size() >= need) return TIDAR_OK;
+  while ((int)s.pages.size() < need) {
+    if (c->free_pages.empty()) return fail(c, TIDAR_ECAPACITY, "KV page pool exhausted");
+    s.pages.push_back(c->free_pages.back());
+    c->free_pages.pop_back();
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_page_table + (size_t)seq * c->pages_per_seq, s.pages.data(), s.pages.size() * sizeof(int),
+                              cudaMemcpyHostToDevice, c->stream));
+  // the source vector may be reallocated by a later call: make the copy complete first
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced) {
+  const tidar_config &cf = c->cfg;
+  if (!seqs || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is already in flight; call tidar_step_wait first");
+  int k = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int q = seqs[i];
+    if (q < 0 || q >= cf.max_batch || !c->seqs[q].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", q);
+    for (int j = 0; j < i; ++j) if (seqs[j] == q) return fail(c, TIDAR_EINVAL, "sequence %d listed twice", q);
+    if (i == 0) k = c->seqs[q].k;
+    else if (c->seqs[q].k != k) return fail(c, TIDAR_EINVAL, "all sequences of a step must share one draft length k");
+    const int f = forced ? forced[i] : 0;
+    if (f < 0 || f > k) return fail(c, TIDAR_EINVAL, "forced acceptance %d outside [0, %d]", f, k);
+    if (need_forced && f == 0) return fail(c, TIDAR_EINVAL, "tidar_step_async needs a forced acceptance length per sequence");
+    if (c->seqs[q].n + 2 * k > cf.max_seq_len)
+      return fail(c, TIDAR_ECAPACITY, "sequence %d: n + 2k = %d exceeds max_seq_len %d", q, c->seqs[q].n + 2 * k, cf.max_seq_len);
+  }
+  for (int i = 0; i < n_seqs; ++i) {
+    int rc = ensure_pages(c, seqs[i], c->seqs[seqs[i]].n + k);
+    if (rc) return rc;
+  }
+  const int T = k * (k + 1), R = n_seqs * T;
+  for (int i = 0; i < n_seqs; ++i) { c->h_stage[i] = seqs[i]; c->h_stage[cf.max_batch + i] = forced ? forced[i] : 0; }
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  {
+    Launch l(c, TIDAR_TC_EMBED);
+    assemble_step_kernel<<<R, 128, 0, c->stream>>>(c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
+                                                   c->d_step_n, c->embed, cf.d_model, c->X);
+  }
+  int rc = forward_rows(c, R, true);
+  if (rc) return rc;
+  {
+    Launch l(c, TIDAR_TC_VERIFY);
+    verify_select_kernel<<<n_seqs, 32, 0, c->stream>>>(c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
+                                                       c->d_step_L, c->d_out);
+  }
+  {
+    Launch l(c, TIDAR_TC_VERIFY);
+    kv_commit_kernel<<<dim3(n_seqs, cf.n_layers), 128, 0, c->stream>>>(c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
+                                                                       (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaGetLastError());
+  c->pending_seqs.assign(seqs, seqs + n_seqs);
+  c->pending = true;
+  c->last_rows = R; c->last_first_pos = -1;
+  // the host tracks lengths without reading the device when L is forced
+  return TIDAR_OK;
+}
+
+int finish_step(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
+  if (!c->pending) return fail(c, TIDAR_EINVAL, "no step in flight");
+  c->pending = false;
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (c->timing) collect_timing(c);
+  const int km = c->cfg.k_max;
+  for (size_t i = 0; i < c->pending_seqs.size(); ++i) {
+    const int L = c->h_pinned[i * (km + 1)];
+    c->seqs[c->pending_seqs[i]].n += L;
+    if (out_n) out_n[i] = L;
+    if (out_tokens) for (int j = 0; j < km; ++j) out_tokens[i * km + j] = j < L ? c->h_pinned[i * (km + 1) + 1 + j] : -1;
+  }
+  return TIDAR_OK;
+}
+
+}  // namespace
+
+// =============================================================================
+extern "C" {
+
+int tidar_arena_bytes(const tidar_config *cfg, size_t *out_bytes) {
+  if (!cfg || !out_bytes) return fail(nullptr, TIDAR_EINVAL, "null argument");
+  std::string why;
+  if (int rc = validate(*cfg, why)) return fail(nullptr, rc, "%s", why.c_str());
+  tidar_ctx tmp; tmp.cfg = *cfg;
+  layout(tmp, nullptr, out_bytes);
+  return TIDAR_OK;
+}
+
+int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, size_t arena_bytes, void *cuda_stream,
+               tidar_ctx **out) {
+  if (!cfg || !w || !arena || !out) return fail(nullptr, TIDAR_EINVAL, "null argument");
+  std::string why;
+  if (int rc = validate(*cfg, why)) return fail(nullptr, rc, "%s", why.c_str());
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return fail(nullptr, TIDAR_ECUDA, "no CUDA device: this library has no CPU path");
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wqkv || !w->wo || !w->ffn_norm || !w->w_gate_up || !w->w_down)
+    return fail(nullptr, TIDAR_EINVAL, "null weight pointer");
+  if ((uintptr_t)arena % 256) return fail(nullptr, TIDAR_EINVAL, "arena must be 256-byte aligned");
+  tidar_ctx *c = new tidar_ctx;
+  c->cfg = *cfg;
+  c->stream = (cudaStream_t)cuda_stream;
+  size_t need = 0;
+  layout(*c, arena, &need);
+  if (need > arena_bytes) { delete c; return fail(nullptr, TIDAR_ENOMEM, "arena has %zu bytes, %zu needed", arena_bytes, need); }
+  c->embed = (const bf16 *)w->embed; c->lm_head = (const bf16 *)w->lm_head; c->final_norm = (const bf16 *)w->final_norm;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->ffn_norm[l] || !w->w_gate_up[l] || !w->w_down[l]) {
+      delete c; return fail(nullptr, TIDAR_EINVAL, "null weight pointer in layer %d", l);
+    }
+    c->attn_norm.push_back((const bf16 *)w->attn_norm[l]); c->wqkv.push_back((const bf16 *)w->wqkv[l]);
+    c->wo.push_back((const bf16 *)w->wo[l]); c->ffn_norm.push_back((const bf16 *)w->ffn_norm[l]);
+    c->wgu.push_back((const bf16 *)w->w_gate_up[l]); c->wdown.push_back((const bf16 *)w->w_down[l]);
+  }
+  c->seqs.resize(cfg->max_batch);
+  // free list in a scrambled order so that page tables are never contiguous
+  c->free_pages.resize(c->n_pages);
+  for (int i = 0; i < c->n_pages; ++i) c->free_pages[i] = i;
+  uint32_t st = 0x9e3779b9u;
+  for (int i = c->n_pages - 1; i > 0; --i) { st = st * 1664525u + 1013904223u; std::swap(c->free_pages[i], c->free_pages[(st >> 8) % (i + 1)]); }
+  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
+  if (e != cudaSuccess) { delete c; return fail(nullptr, TIDAR_ECUDA, "cudaHostAlloc: %s", cudaGetErrorString(e)); }
+  c->h_stage = c->h_pinned + (size_t)cfg->max_batch * (cfg->k_max + 1);
+  e = cudaMemsetAsync(c->d_seq_len, 0, cfg->max_batch * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_page_table, 0, (size_t)cfg->max_batch * c->pages_per_seq * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return fail(nullptr, TIDAR_ECUDA, "arena set-up: %s", cudaGetErrorString(e)); }
+  *out = c;
+  return TIDAR_OK;
+}
+
+int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_prompt, int32_t k, int32_t *out_first) {
+  if (!c) return TIDAR_EINVAL;
+  const tidar_config &cf = c->cfg;
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (seq < 0 || seq >= cf.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
+  if (!prompt || n_prompt < 1) return fail(c, TIDAR_EINVAL, "empty prompt");
+  if (k < 1 || k > cf.k_max) return fail(c, TIDAR_EINVAL, "k must be in [1, k_max]");
+  if (n_prompt + 2 * k > cf.max_seq_len) return fail(c, TIDAR_ECAPACITY, "n_prompt + 2k = %d exceeds max_seq_len %d", n_prompt + 2 * k, cf.max_seq_len);
+  for (int i = 0; i < n_prompt; ++i)
+    if (prompt[i] < 0 || prompt[i] >= cf.vocab) return fail(c, TIDAR_EINVAL, "prompt id %d at %d out of range", prompt[i], i);
+  SeqState &s = c->seqs[seq];
+  for (int p : s.pages) c->free_pages.push_back(p);
+  s.pages.clear(); s.active = false; s.n = 0; s.k = k;
+  if (int rc = ensure_pages(c, seq, n_prompt + k)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_prompt, prompt, (size_t)n_prompt * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  const int total = n_prompt + k;
+  const int last_rows = std::min(total, c->R_cap);
+  int row0 = 0;
+  while (row0 < total) {
+    const bool last = row0 >= total - last_rows;
+    const int rows = last ? total - row0 : std::min(c->R_cap, total - last_rows - row0);
+    {
+      Launch l(c, TIDAR_TC_EMBED);
+      assemble_prefill_kernel<<<rows, 128, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
+                                                           cf.d_model, c->X);
+    }
+    if (int rc = forward_rows(c, rows, last)) return rc;
+    if (last) {
+      Launch l(c, TIDAR_TC_VERIFY);
+      prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, n_prompt - 1 - row0, k, cf.k_max, seq, n_prompt, c->d_block,
+                                                     c->d_seq_len, c->d_out);
+      c->last_rows = rows; c->last_first_pos = row0;
+    }
+    row0 += rows;
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  CUDA_TRY(c, cudaGetLastError());
+  if (c->timing) collect_timing(c);
+  s.n = n_prompt; s.active = true;
+  if (out_first) *out_first = c->h_pinned[0];
+  return TIDAR_OK;
+}
+
+int tidar_step(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, const int32_t *forced, int32_t *out_tokens, int32_t *out_n) {
+  if (!c) return TIDAR_EINVAL;
+  if (int rc = enqueue_step(c, seqs, n_seqs, forced, false)) return rc;
+  return finish_step(c, out_tokens, out_n);
+}
+
+int tidar_step_async(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, const int32_t *forced) {
+  if (!c) return TIDAR_EINVAL;
+  if (!forced) return fail(c, TIDAR_EINVAL, "tidar_step_async needs forced acceptance lengths");
+  return enqueue_step(c, seqs, n_seqs, forced, true);
+}
+
+int tidar_step_wait(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
+  if (!c) return TIDAR_EINVAL;
+  return finish_step(c, out_tokens, out_n);
+}
+
+int tidar_free(tidar_ctx *c) {
+  if (!c) return TIDAR_EINVAL;
+  cudaStreamSynchronize(c->stream);
+  for (auto &t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+  if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  delete c;
+  return TIDAR_OK;
+}
+
+const char *tidar_last_error(const tidar_ctx *c) { return c ? c->err.c_str() : g_init_error.c_str(); }
+
+int tidar_seq_len(const tidar_ctx *c, int32_t seq) {
+  if (!c || seq < 0 || seq >= c->cfg.max_batch || !c->seqs[seq].active) return TIDAR_EINVAL;
+  return c->seqs[seq].n;
+}
+
+int64_t tidar_launch_count(const tidar_ctx *c) { return c ? c->launches : -1; }
+
+int tidar_debug_set_block(tidar_ctx *c, int32_t seq, const int32_t *block) {
+  if (!c || !block) return TIDAR_EINVAL;
+  if (seq < 0 || seq >= c->cfg.max_batch || !c->seqs[seq].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", seq);
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_block + (size_t)seq * c->cfg.k_max, block, c->seqs[seq].k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_block(tidar_ctx *c, int32_t seq, int32_t *block) {
+  if (!c || !block) return TIDAR_EINVAL;
+  if (seq < 0 || seq >= c->cfg.max_batch || !c->seqs[seq].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", seq);
+  CUDA_TRY(c, cudaMemcpyAsync(block, c->d_block + (size_t)seq * c->cfg.k_max, c->seqs[seq].k * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_last_rows(const tidar_ctx *c, int32_t *n_rows, int32_t *first_pos) {
+  if (!c) return TIDAR_EINVAL;
+  if (n_rows) *n_rows = c->last_rows;
+  if (first_pos) *first_pos = c->last_first_pos;
+  return TIDAR_OK;
+}
+
+static int check_rows(tidar_ctx *c, int row0, int n) {
+  if (row0 < 0 || n < 1 || row0 + n > c->last_rows) return fail(c, TIDAR_EINVAL, "rows [%d, %d) outside the last pass (%d rows)", row0, row0 + n, c->last_rows);
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_logits(tidar_ctx *c, int32_t row0, int32_t n, float *out) {
+  if (!c || !out) return TIDAR_EINVAL;
+  if (!c->dbg_logits) return fail(c, TIDAR_EINVAL, "context was created without debug bit 0");
+  if (int rc = check_rows(c, row0, n)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(out, c->dbg_logits + (size_t)row0 * c->cfg.vocab, (size_t)n * c->cfg.vocab * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_hidden(tidar_ctx *c, int32_t layer, int32_t row0, int32_t n, float *out) {
+  if (!c || !out) return TIDAR_EINVAL;
+  if (!c->dbg_hidden) return fail(c, TIDAR_EINVAL, "context was created without debug bit 0");
+  if (layer < 0 || layer > c->cfg.n_layers) return fail(c, TIDAR_EINVAL, "layer out of range");
+  if (int rc = check_rows(c, row0, n)) return rc;
+  const size_t d = c->cfg.d_model;
+  CUDA_TRY(c, cudaMemcpyAsync(out, c->dbg_hidden + ((size_t)layer * c->R_cap + row0) * d, (size_t)n * d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_argmax(tidar_ctx *c, int32_t row0, int32_t n, int32_t *out) {
+  if (!c || !out) return TIDAR_EINVAL;
+  if (int rc = check_rows(c, row0, n)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(out, c->d_arg_idx + row0, (size_t)n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_kv(tidar_ctx *c, int32_t seq, int32_t layer, int32_t pos0, int32_t npos, uint16_t *k_out, uint16_t *v_out) {
+  if (!c || !k_out || !v_out) return TIDAR_EINVAL;
+  if (seq < 0 || seq >= c->cfg.max_batch || !c->seqs[seq].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", seq);
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, TIDAR_EINVAL, "layer out of range");
+  const int backed = (int)c->seqs[seq].pages.size() * c->cfg.page_size;
+  if (pos0 < 0 || npos < 1 || pos0 + npos > backed) return fail(c, TIDAR_EINVAL, "positions [%d, %d) not backed by pages (%d)", pos0, pos0 + npos, backed);
+  const size_t per = (size_t)c->cfg.n_kv_heads * c->cfg.head_dim;
+  const bf16 *Kp = c->kv + (size_t)(2 * layer) * c->pool_stride, *Vp = Kp + c->pool_stride;
+  for (int p = 0; p < npos; p += 256) {
+    const int np = std::min(256, npos - p);
+    bf16 *ko = c->dbg_kv, *vo = c->dbg_kv + 256 * per;
+    kv_gather_kernel<<<dim3(np, c->cfg.n_kv_heads), 64, 0, c->stream>>>(Kp, Vp, geom(c), seq, pos0 + p, ko, vo);
+    CUDA_TRY(c, cudaMemcpyAsync(k_out + (size_t)p * per, ko, np * per * 2, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(v_out + (size_t)p * per, vo, np * per * 2, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  }
+  return TIDAR_OK;
+}
+
+int tidar_debug_set_timing(tidar_ctx *c, int32_t on) {
+  if (!c) return TIDAR_EINVAL;
+  c->timing = on != 0;
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_timing(tidar_ctx *c, float *ms) {
+  if (!c || !ms) return TIDAR_EINVAL;
+  for (int i = 0; i < TIDAR_TC_COUNT; ++i) ms[i] = c->class_ms[i];
+  return TIDAR_OK;
+}
+
+int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                    int32_t pages_per_seq, const int32_t *seq_len, const void *k_local, const void *v_local, void *out,
+                    int32_t n_seqs, int32_t k) {
+  if (!c) return TIDAR_EINVAL;
+  if (!q || !k_pages || !v_pages || !page_table || !seq_len || !k_local || !v_local || !out) return fail(c, TIDAR_EINVAL, "null argument");
+  if (k < 1 || k > c->cfg.k_max || n_seqs < 1 || n_seqs * k * (k + 1) > c->R_cap) return fail(c, TIDAR_EINVAL, "n_seqs * k(k+1) exceeds the context's row capacity");
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  const int R = n_seqs * k * (k + 1);
+  {
+    Launch l(c, TIDAR_TC_EMBED);
+    attn_meta_kernel<<<(R + 127) / 128, 128, 0, c->stream>>>(c->meta, seq_len, k, R);
+  }
+  KvGeom g{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, pages_per_seq, page_table};
+  launch_attention(c, (const bf16 *)q, (const bf16 *)k_pages, (const bf16 *)v_pages, g, (const bf16 *)k_local, (const bf16 *)v_local,
+                   (bf16 *)out, R);
+  CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
+}  // extern "C"

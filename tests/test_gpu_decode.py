@@ -1,0 +1,244 @@
+"""CUDA path vs oracle on the decode step, through the C ABI (needs a B200)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tidar_oracle as O
+from tests.helpers import MARGIN, TOL_LOGITS, make_model, oracle_cfg, prompt_ids, top1_margin
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [1]
+
+
+def _gpu(sh, wt, impl, k_max=None, debug=1, max_batch=1, max_seq_len=512):
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    packed = pack_weights(wt, "cuda:0")
+    return Tidar(sh, packed, k_max=k_max or sh.k, max_batch=max_batch, max_seq_len=max_seq_len, debug=debug, impl=impl)
+
+
+@pytest.fixture(scope="module", params=[True, False], ids=["tied", "untied"])
+def tiny(request):
+    sh, wt = make_model("tiny", tied=request.param)
+    return sh, wt, oracle_cfg(sh), O.weights_to_f64(wt), prompt_ids(sh)
+
+
+def _compare_pass(t, fo, rows, tol=TOL_LOGITS):
+    """logits / hidden of the last GPU pass against an oracle ForwardOut restricted to rows."""
+    n_rows, _ = t.last_rows()
+    assert n_rows == len(rows)
+    lg = t.logits(0, n_rows)
+    ref = fo.logits[rows]
+    assert np.isfinite(lg).all()
+    assert np.abs(lg - ref).max() <= tol
+    for l in range(len(fo.hidden)):
+        h = t.hidden(l, 0, n_rows)
+        assert np.abs(h - fo.hidden[l][rows]).max() <= tol
+    ids = t.argmax(0, n_rows)
+    np.testing.assert_array_equal(ids, lg.argmax(-1))          # fused argmax == argmax of its own logits
+    sure = top1_margin(ref) > MARGIN
+    np.testing.assert_array_equal(ids[sure], ref.argmax(-1)[sure])
+    return lg, ids
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_prefill_and_teacher_forced_steps(tiny, impl):
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    t = _gpu(sh, wt, impl)
+    first = t.prefill(0, prompt, k)
+    st, c, fo = O.prefill(cfg, w, prompt, k, return_forward=True)
+    lg, ids = _compare_pass(t, fo, np.arange(len(prompt) + k))
+    n = len(prompt)
+    assert first == int(lg[n - 1].argmax())
+    blk = t.get_block(0, k)
+    assert blk == [int(lg[n - 1].argmax())] + [int(x) for x in lg[n + 1:n + k].argmax(-1)]
+    # KV of the prompt
+    for l in range(cfg.n_layers):
+        from paper_2511_08923_b200 import bf16_bits_to_f32
+        kk, vv = t.kv(0, l, 0, n)
+        assert np.abs(bf16_bits_to_f32(kk) - st.k_cache[l]).max() <= TOL_LOGITS
+        assert np.abs(bf16_bits_to_f32(vv) - st.v_cache[l]).max() <= TOL_LOGITS
+    # decode steps, teacher-forced: the GPU gets the oracle's block before every step
+    ar = O.ar_generate(cfg, w, prompt, 40)
+    for s in range(6):
+        e = st.n - n
+        if s % 3 == 1:                       # perfect drafts -> L = k
+            st.block[1:] = ar[e + 1:e + k]
+        elif s % 3 == 2:                     # two right, then wrong
+            st.block[1:] = ar[e + 1:e + k]
+            st.block[3] = (st.block[3] + 1) % (sh.vocab - 1)
+        t.set_block(0, st.block)
+        block_before = st.block.copy()
+        n_before = st.n
+        so = O.step(cfg, w, st)
+        toks, Ls = t.step([0])
+        lg, ids = _compare_pass(t, so.fwd, np.arange(k * (k + 1)))
+        # integer logic, bit-exact given the GPU's own argmax ids
+        tg = ids[:k]
+        L_ref = O.accept_length(block_before, tg)
+        assert Ls[0] == L_ref
+        assert toks[0] == [int(x) for x in block_before[1:L_ref]] + [int(tg[L_ref - 1])]
+        nxt = O.select_next(L_ref, tg, ids[k:].reshape(k, k))
+        assert t.get_block(0, k) == [int(x) for x in nxt]
+        assert t.seq_len(0) == n_before + L_ref
+        if (top1_margin(so.fwd.logits[:k]) > MARGIN).all():
+            assert Ls[0] == so.L and toks[0] == so.emitted
+        elif Ls[0] != so.L:                   # a low-margin row flipped: the two states part ways here
+            break
+    t.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_free_running_generation_matches_ar(tiny, impl):
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    ar = O.ar_generate(cfg, w, prompt, sh.max_new_tokens)
+    t = _gpu(sh, wt, impl)
+    out = [t.prefill(0, prompt, k)]
+    Ls = []
+    while len(out) < sh.max_new_tokens:
+        toks, L = t.step([0])
+        out.extend(toks[0]); Ls.append(L[0])
+    out = out[:sh.max_new_tokens]
+    # compare up to the first position where the oracle itself is not sure
+    fo = O.causal_forward(cfg, w, list(prompt) + ar)
+    m = top1_margin(fo.logits[len(prompt) - 1:len(prompt) - 1 + sh.max_new_tokens])
+    unsure = np.nonzero(m <= MARGIN)[0]
+    upto = int(unsure[0]) if len(unsure) else sh.max_new_tokens
+    assert out[:upto] == ar[:upto]
+    assert all(1 <= L <= k for L in Ls)
+    assert t.seq_len(0) == len(prompt) + sum(Ls)
+    t.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_acceptance_scan_all_patterns(tiny, impl):
+    """Every agree/disagree pattern of the k-1 drafts, driven through the real step."""
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    t = _gpu(sh, wt, impl, debug=0)
+    first = t.prefill(0, prompt, k)
+    blk = t.get_block(0, k)
+    for pattern in itertools.product([True, False], repeat=k - 1):
+        # targets of causal slot 0 do not depend on drafts; build slot by slot
+        block = [blk[0]]
+        for i in range(1, k):
+            t.prefill(0, prompt, k)
+            t.set_block(0, block + [sh.mask_token_id] * (k - len(block)))
+            toks_i, L_i = t.step([0], forced=[i])
+            tgt = toks_i[0][-1]                          # verified prediction after i slots
+            block.append(tgt if pattern[i - 1] else (tgt + 1) % (sh.vocab - 1))
+        t.prefill(0, prompt, k)
+        t.set_block(0, block)
+        toks, L = t.step([0])
+        expect = next((i for i, ok in enumerate(pattern) if not ok), k - 1) + 1
+        assert L[0] == expect, (pattern, block)
+        assert toks[0][:expect - 1] == block[1:expect]
+    t.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_forced_acceptance_and_poisoned_eviction(tiny, impl):
+    """Forced L commits exactly L slots; NaN-filling evicted slots changes nothing."""
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    runs = []
+    for debug in (1, 3):
+        t = _gpu(sh, wt, impl, debug=debug)
+        t.prefill(0, prompt, k)
+        rec = []
+        for L in (1, 3, 2, 4, 1):
+            toks, Ls = t.step([0], forced=[L])
+            assert Ls == [L] and len(toks[0]) == L
+            rec.append((toks[0], t.get_block(0, k), t.logits(0, k * (k + 1)).copy()))
+        n = t.seq_len(0)
+        assert n == len(prompt) + 11
+        rec.append([t.kv(0, l, 0, n) for l in range(cfg.n_layers)])
+        runs.append(rec)
+        t.close()
+    for a, b in zip(runs[0][:-1], runs[1][:-1]):
+        assert a[0] == b[0] and a[1] == b[1]
+        np.testing.assert_array_equal(a[2], b[2])
+    for (k0, v0), (k1, v1) in zip(runs[0][-1], runs[1][-1]):
+        np.testing.assert_array_equal(k0, k1); np.testing.assert_array_equal(v0, v1)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_committed_kv_is_exact_and_never_rewritten(tiny, impl):
+    """The cache after decoding equals, bit for bit, what a fresh first pass over the
+    final sequence writes for layer 0 (row-wise deterministic kernels), stays within
+    tolerance of the oracle for every layer, and committed rows never change later."""
+    from paper_2511_08923_b200 import bf16_bits_to_f32
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    t = _gpu(sh, wt, impl, debug=0)
+    seq = list(prompt) + [t.prefill(0, prompt, k)]
+    snaps = []
+    for L in (2, 4, 1, 3):
+        toks, _ = t.step([0], forced=[L])
+        seq.extend(toks[0])
+        n = t.seq_len(0)
+        snaps.append((n, [t.kv(0, l, 0, n) for l in range(cfg.n_layers)]))
+    n_final = t.seq_len(0)
+    final = [t.kv(0, l, 0, n_final) for l in range(cfg.n_layers)]
+    for n, kv in snaps:
+        for l in range(cfg.n_layers):
+            np.testing.assert_array_equal(kv[l][0], final[l][0][:n]); np.testing.assert_array_equal(kv[l][1], final[l][1][:n])
+    ref = O.causal_forward(cfg, w, seq[:n_final])
+    for l in range(cfg.n_layers):
+        assert np.abs(bf16_bits_to_f32(final[l][0]) - ref.k_new[l]).max() <= TOL_LOGITS
+        assert np.abs(bf16_bits_to_f32(final[l][1]) - ref.v_new[l]).max() <= TOL_LOGITS
+    # replay: a first pass over the same tokens on a fresh sequence slot
+    t2 = _gpu(sh, wt, impl, debug=0)
+    t2.prefill(0, seq[:n_final], k)
+    k0, v0 = t2.kv(0, 0, 0, n_final)
+    np.testing.assert_array_equal(k0, final[0][0]); np.testing.assert_array_equal(v0, final[0][1])
+    t.close(); t2.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_batched_step_equals_single_sequence_steps(impl):
+    sh, wt = make_model("tiny", tied=False)
+    k = sh.k
+    prompts = [prompt_ids(sh, n, seed=s) for n, s in ((64, 0), (37, 5), (1, 6))]
+    single = []
+    for p in prompts:
+        t = _gpu(sh, wt, impl, debug=0)
+        out = [t.prefill(0, p, k)]
+        for L in (2, 1, 4):
+            out.extend(t.step([0], forced=[L])[0][0])
+        single.append(out); t.close()
+    t = _gpu(sh, wt, impl, debug=0, max_batch=3)
+    outs = [[t.prefill(i, p, k)] for i, p in enumerate(prompts)]
+    for L in (2, 1, 4):
+        toks, _ = t.step([0, 1, 2], forced=[L, L, L])
+        for i in range(3):
+            outs[i].extend(toks[i])
+    assert outs == single
+    t.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_errors_are_reported_before_launch(impl):
+    from paper_2511_08923_b200 import TidarError
+    sh, wt = make_model("tiny")
+    t = _gpu(sh, wt, impl, debug=0, max_seq_len=80)
+    with pytest.raises(TidarError) as e:
+        t.step([0])
+    assert e.value.code == -1
+    with pytest.raises(TidarError) as e:
+        t.prefill(0, prompt_ids(sh, 73), 4)             # 73 + 8 > 80
+    assert e.value.code == -2
+    t.prefill(0, prompt_ids(sh, 70), 4)
+    t.step([0], forced=[2])
+    with pytest.raises(TidarError) as e:                 # 72 + 8 = 80 fits, then 73.. does not
+        t.step([0], forced=[1]); t.step([0], forced=[1])
+    assert e.value.code == -2
+    with pytest.raises(TidarError):
+        t.prefill(0, [5000], 4)
+    with pytest.raises(TidarError):
+        t.step([0], forced=[9])
+    t.close()
