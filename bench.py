@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the TiDAR decode step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b|1.5b|tiny] [--impl ours|reference]
+
+A "step" is one pass of the whole decode path (slot assembly, every layer, LM
+head with argmax, draft/verify/select, KV commit) for one sequence.  Prints ONE
+JSON line.  Metric: decode tokens/s under a seeded acceptance-length schedule
+(mean 8 at k = 16); the step cost does not depend on the acceptance length, so
+the per-length table is tokens/s = L / latency.
+
+``--impl reference`` times the CPU oracle (the only reference this method has) on
+a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from tidar_synth import CONFIGS, acceptance_schedule, gen_model_weights, gen_token_ids, tensor_id
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+SCHEDULE_SEED = 1234
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------
+# algorithmic cost of one step (per sequence)
+# ----------------------------------------------------------------------------
+def step_cost(sh, k, n, n_layers=None):
+    """Algorithmic bytes and flops of one decode step with n cached positions.
+
+    bytes: every projection weight and the LM head once (bf16) + the K/V of the n
+    cached positions once per layer.  flops: 2*T*params for the projections +
+    4*T*Hq*hd*(keys visible per row) for attention.
+    """
+    T = k * (k + 1)
+    L = n_layers or sh.n_layers
+    per_layer = (sh.d_model * (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim + sh.n_q_heads * sh.head_dim * sh.d_model
+                 + 3 * sh.d_model * sh.d_ffn)
+    params = L * per_layer + sh.vocab * sh.d_model
+    kv_bytes = n * L * 2 * sh.n_kv_heads * sh.head_dim * 2
+    # keys per row: causal j sees n+j+1, mask (b, .) sees n+b+1+k
+    keys = sum(n + j + 1 for j in range(k)) + sum(k * (n + b + 1 + k) for b in range(k))
+    attn_flops = L * 4 * sh.n_q_heads * sh.head_dim * keys
+    return {"T": T, "params": params, "weight_bytes": 2 * params, "kv_bytes": kv_bytes,
+            "gemm_flops": 2 * T * params, "attn_flops": attn_flops,
+            "bytes": 2 * params + kv_bytes, "flops": 2 * T * params + attn_flops}
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx, self.p = gpu_index, None
+
+    def __enter__(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.p = None
+        return self
+
+    def __exit__(self, *a):
+        self.out = ""
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.out, _ = self.p.communicate(timeout=5)
+            except Exception:
+                self.p.kill()
+
+    def summary(self):
+        sm, mx, reasons, pw = [], [], set(), []
+        for line in self.out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        # samples under load = upper half of the clock samples' power
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_max": max(pw)}
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle on a bounded sample
+# ----------------------------------------------------------------------------
+def oracle_sample(sh, k, n, with_head=True, rows=None):
+    """Time the oracle on ONE layer (+ the LM head) of one decode step; extrapolate a step.
+
+    The weights are the generator's (layer 0 and the LM head); the embedding table is
+    restricted to the ids in use (ids remapped), the cache holds seeded random K/V.
+    """
+    from oracle import tidar_oracle as O
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = gen_model_weights(sh.reduced(1), device=dev)
+    lay = {kk: (vv if kk == "index" else vv.cpu()) for kk, vv in w["layers"][0].items()}
+    block = gen_token_ids(sh.seed, tensor_id("drafts"), k, sh.vocab - 1).numpy().astype(np.int64)
+    used = np.unique(np.concatenate([block, [sh.mask_token_id]]))
+    remap = {int(u): i for i, u in enumerate(used)}
+    small_embed = w["embed"][torch.as_tensor(used, device=w["embed"].device)].cpu()
+    wd = {"embed": small_embed, "final_norm": w["final_norm"].cpu(), "lm_head": w["lm_head"].cpu(), "layers": [lay]}
+    t0 = time.perf_counter()
+    w64 = O.weights_to_f64(wd)
+    t_upcast = time.perf_counter() - t0
+    cfg = O.OracleConfig(1, sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.d_ffn, sh.vocab, sh.rope_theta,
+                         sh.rms_eps, remap[sh.mask_token_id], 1.0)
+    rng = np.random.default_rng(sh.seed)
+    st = O.OracleState(n=n, k_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim))],
+                       v_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim))],
+                       block=np.array([remap[int(b)] for b in block]))
+    # layer part: a pass without the head (logit_rows empty), head part: the difference
+    T = k * (k + 1)
+    _, _, _, pos = O.slot_layout(n, k)
+    ids = np.concatenate([st.block, np.full(k * k, cfg.mask_token_id, dtype=np.int64)])
+    mask = O.build_decode_mask(n, k)
+
+    def run(head):
+        t0 = time.perf_counter()
+        O.forward(cfg, w64, ids, pos, mask, st.k_cache, st.v_cache, logit_rows=None if head else np.array([], dtype=np.int64))
+        return time.perf_counter() - t0
+    return run, t_upcast
+
+
+def oracle_step_seconds(sh, t_layer, t_head):
+    return sh.n_layers * t_layer + t_head
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+# ----------------------------------------------------------------------------
+def run_reference(args, sh, k, n0):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sched = acceptance_schedule(SCHEDULE_SEED, args.steps + args.warmup, k).numpy()
+    run, _ = oracle_sample(sh, k, n0)
+    t_l = run(False)
+    t_full = run(True)
+    t_h = max(t_full - t_l, 0.0)
+    budget = 150.0
+    total_steps = args.steps + args.warmup
+    do_head = total_steps * (t_l + t_h) <= budget
+    layer_s, head_s = [], []
+    for s in range(total_steps):
+        if do_head:
+            a = run(False); b = run(True)
+            if s >= args.warmup:
+                layer_s.append(a); head_s.append(max(b - a, 0.0))
+        elif total_steps * t_l <= budget:
+            a = run(False)
+            if s >= args.warmup:
+                layer_s.append(a); head_s.append(t_h)
+        else:
+            if s >= args.warmup:
+                layer_s.append(t_l); head_s.append(t_h)
+    step_s = [oracle_step_seconds(sh, a, b) for a, b in zip(layer_s, head_s)]
+    L = sched[args.warmup:]
+    value = float(L.sum() / sum(step_s))
+    sample = (f"per step: one of {sh.n_layers} layers" + (" + the full LM head" if do_head else " (LM head timed once)") +
+              f" of one decode step (k={k}, {k*(k+1)} slots, n={n0}); step time = n_layers*layer + head")
+    if not do_head and total_steps * t_l > budget:
+        sample = "calibration pass only (one layer + LM head timed once; requested steps exceed the time bound); " + sample
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(step_s) / len(step_s),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(sh, k, n0, 1),
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(sh, k, n0, batch):
+    return {"workload": f"TiDAR decode step, {sh.name}-class decoder ({sh.n_layers} layers, d_model {sh.d_model}, "
+                        f"{sh.n_q_heads}/{sh.n_kv_heads} heads, head_dim {sh.head_dim}, ffn {sh.d_ffn}, vocab {sh.vocab}), "
+                        f"bf16 random-init seed {sh.seed}, batch {batch}, prompt {n0} random ids, k={k} ({k*(k+1)} slots/step), greedy",
+            "acceptance": f"seeded truncated-geometric schedule (seed {SCHEDULE_SEED}, p=0.8969, mean 8 at k=16)",
+            "l2": "inputs larger than L2: each step streams every weight once (>> 126 MB)",
+            "k": k, "prompt_len": n0, "batch": batch}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b", choices=list(CONFIGS))
+    ap.add_argument("--kernels", type=int, default=None, help="library impl: 0 tensor-core, 1 replay (diagnostic)")
+    ap.add_argument("--layers", type=int, default=None, help="reduced-depth twin (diagnostics only; not a bench value)")
+    ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--per-l-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    sh = CONFIGS[args.workload]
+    if args.layers:
+        sh = sh.reduced(args.layers)
+    k = args.k or sh.k
+    n0 = sh.prompt_len
+    if args.impl == "reference":
+        run_reference(args, sh, k, n0)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    impl = args.kernels if args.kernels is not None else DEFAULT_IMPL
+    wt = gen_model_weights(sh, device=dev)
+    packed = pack_weights(wt, dev)
+    del wt
+    torch.cuda.empty_cache()
+    stream = torch.cuda.Stream(device=dev)
+    n_steps_total = args.warmup + 2 * args.steps + 8 + k * args.per_l_steps
+    t = Tidar(sh, packed, k_max=k, max_batch=1, max_seq_len=n0 + (n_steps_total + 4) * k + 2 * k + 64, impl=impl,
+              device=dev, stream=stream)
+    prompt = gen_token_ids(sh.seed, tensor_id("prompt"), n0, sh.vocab - 1).numpy()
+    t.prefill(0, prompt, k)
+    sched = acceptance_schedule(SCHEDULE_SEED, args.warmup + 2 * args.steps, k).numpy()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps, CUDA events on the library's stream -----
+    si = 0
+    for _ in range(args.warmup):
+        t.step_async([0], [int(sched[si])]); t.step_wait(); si += 1
+    n_start = t.seq_len(0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = t.launch_count()
+    barrier()
+    with ClockSampler(local) as clk:
+        with torch.cuda.stream(stream):
+            ev0.record(stream)
+        tokens = 0
+        for _ in range(args.steps):
+            t.step_async([0], [int(sched[si])]); _, L = t.step_wait(); tokens += L[0]; si += 1
+        with torch.cuda.stream(stream):
+            ev1.record(stream)
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = t.launch_count() - launches0
+    n_mid = (n_start + t.seq_len(0)) // 2
+    clocks = clk.summary()
+
+    # ---- end to end through tidar_step with host buffers (wall clock) --------------
+    barrier()
+    w0 = time.perf_counter()
+    tokens_e2e = 0
+    for _ in range(args.steps):
+        _, L = t.step([0], [int(sched[si])]); tokens_e2e += L[0]; si += 1
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - w0
+
+    # ---- per-class kernel time (CUDA events around every launch) ---------------------
+    t.set_timing(True)
+    cls = {}
+    n_t = 4
+    for _ in range(n_t):
+        t.step([0], [8 if k >= 8 else k])
+        for kk, v in t.timing().items():
+            cls[kk] = cls.get(kk, 0.0) + v / n_t
+    t.set_timing(False)
+
+    # ---- per acceptance length -----------------------------------------------------------
+    per_L = {}
+    for L in range(1, k + 1):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(args.per_l_steps):
+            t.step_async([0], [L]); t.step_wait()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / args.per_l_steps
+        per_L[str(L)] = {"ms_per_step": round(ms, 4), "tokens_per_s": round(L / ms * 1e3, 1)}
+
+    if world > 1:
+        tt = torch.tensor([ms_total, e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total, e2e_s = float(tt[0]), float(tt[1])
+        tk = torch.tensor([tokens, tokens_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        tokens, tokens_e2e = float(tk[0]), float(tk[1])
+
+    if rank == 0:
+        pk, pk_src = peaks()
+        ms_step = ms_total / args.steps
+        cost = step_cost(sh, k, n_mid)
+        t_hbm = cost["bytes"] / (pk["hbm_gbs"] * 1e9) * 1e3
+        t_tensor = cost["flops"] / (pk["bf16_tflops_sustained"] * 1e12) * 1e3
+        t_hbm_nom = cost["bytes"] / (NOMINAL["hbm_gbs"] * 1e9) * 1e3
+        t_tensor_nom = cost["flops"] / (NOMINAL["bf16_tflops"] * 1e12) * 1e3
+        gemm_ms = cls.get("gemm", 0.0) + cls.get("lmhead", 0.0)
+        tensor_bound = t_tensor >= t_hbm
+        if tensor_bound:
+            ach = cost["gemm_flops"] / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+            roof = {"bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+        else:
+            ach = cost["weight_bytes"] / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+            roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+        roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": TRAFFIC_NOTE.get(args.workload),
+                     "kernel": "projection GEMMs (QKV, O, gate/up, down, LM head) summed over one step",
+                     "peak_source": pk_src + (" (sustained bf16)" if tensor_bound else " (copy bandwidth)"),
+                     "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {a: round(b, 4) for a, b in cls.items()}})
+        line = {"metric": "decode_tokens_per_s", "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(sh, k, n0, 1), "clocks": clocks,
+                "e2e": {"value": tokens_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": 8, "d2h_bytes_per_step": 4 * (k + 1),
+                        "ms_per_step": 1e3 * e2e_s / args.steps},
+                "gpu_launches": int(launches),
+                "roofline": roof,
+                "step_roofline": {"bytes": cost["bytes"], "flops": cost["flops"], "n_cached": n_mid,
+                                  "t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "frac_measured_peaks": max(t_hbm, t_tensor) / ms_step,
+                                  "frac_nominal_peaks": max(t_hbm_nom, t_tensor_nom) / ms_step, "peaks": pk, "peak_source": pk_src},
+                "mean_accept_len": tokens / (args.steps * world), "per_accept_len": per_L,
+                "kernels": "tcgen05" if impl == 0 else "replay (fp32 CUDA cores)",
+                "paper_context": "paper reports 4.71x (1.5B) / 5.91x (8B) tokens/s over AR on one H100; no absolute figure"}
+        if not args.no_cpu_baseline:
+            run, _ = oracle_sample(sh, k, n0)
+            t_l = run(False); t_f = run(True)
+            step_s = oracle_step_seconds(sh, t_l, max(t_f - t_l, 0.0))
+            mean_L = float(sched.mean())
+            line["cpu_baseline"] = {"value": mean_L / step_s, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"one of {sh.n_layers} layers + the full LM head of one decode step (k={k}, n={n0}), "
+                                              f"float64 NumPy; step = n_layers*layer + head = {step_s:.1f} s"}
+        print(json.dumps(line))
+    t.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+DEFAULT_IMPL = 1
+# dram bytes per step of the projection kernels from an ncu capture (see profiles/); None until captured
+TRAFFIC_NOTE = {}
+
+if __name__ == "__main__":
+    main()
