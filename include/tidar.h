@@ -180,6 +180,33 @@ int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const vo
                     const void *k_local, const void *v_local, void *out,
                     int32_t n_seqs, int32_t k);
 
+/* ---- structured-mask attention for callers that cannot allocate ---------------------
+ * (The paper has no counterpart: this is a packaging variant of tidar_attention.)
+ * Same computation, same tensor layouts and same mask as tidar_attention, but it needs
+ * no context and no arena: the shapes come as plain arguments and the per-row
+ * visibility table, which tidar_attention keeps in the caller-allocated arena, lives in
+ * a fixed table built into the library image.  It is meant for hosts that hold device
+ * tensors but may not call an allocator where they need attention: a server whose
+ * memory pool belongs wholly to another component, a latency-critical loop (cudaMalloc
+ * may stall every stream of the device), a plug-in that is handed buffers only.
+ * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   - Limit: n_seqs * k * (k+1) <= 4352 rows (16 sequences at k = 16); beyond that the
+ *     call returns TIDAR_ECAPACITY and launches nothing.  page_size is 64.
+ *   - Each GPU that loads the library holds the table (85 KiB) until the process exits.
+ *   - The first call on a device looks up the table's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on one device share the table and each call rewrites the entries it uses,
+ *     so nothing needs clearing; but two calls whose kernels may overlap on the GPU
+ *     (different streams, no ordering between them) race on it.  Serialise them.
+ *   - Work is enqueued on cuda_stream (a cudaStream_t, NULL = default) of the current
+ *     device; the call does not synchronise.  All data pointers are DEVICE pointers.
+ * Errors: TIDAR_EINVAL, TIDAR_ECAPACITY, TIDAR_ECUDA; message via tidar_last_error(NULL). */
+int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages,
+                           const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
+                           const void *k_local, const void *v_local, void *out,
+                           int32_t n_seqs, int32_t k, int32_t n_q_heads, int32_t n_kv_heads,
+                           int32_t head_dim, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -78,6 +78,7 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_debug_set_timing": (C.c_int, [ctxp, I32]),
         "tidar_debug_get_timing": (C.c_int, [ctxp, P(C.c_float)]),
         "tidar_attention": (C.c_int, [ctxp, VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32]),
+        "tidar_attention_static": (C.c_int, [VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -258,6 +259,23 @@ class Tidar:
         self._check(self.lib.tidar_attention(
             self.ctx, q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), page_table.data_ptr(), page_table.shape[1],
             seq_len.data_ptr(), k_local.data_ptr(), v_local.data_ptr(), out.data_ptr(), n_seqs, k))
+
+
+def attention_static(q, k_pages, v_pages, page_table, seq_len, k_local, v_local, out, n_seqs: int, k: int,
+                     n_q_heads: int, n_kv_heads: int, head_dim: int, stream: Optional[torch.cuda.Stream] = None):
+    """tidar_attention_static: the attention of a decode step for callers that cannot allocate.
+
+    Needs no :class:`Tidar` context and no arena; all tensors are caller-owned device
+    tensors in the layouts of :meth:`Tidar.attention`.  At most 4352 rows
+    (``n_seqs * k * (k+1)``); calls that may overlap on the GPU must be serialised.
+    """
+    lib = load()
+    rc = lib.tidar_attention_static(q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), page_table.data_ptr(),
+                                    page_table.shape[1], seq_len.data_ptr(), k_local.data_ptr(), v_local.data_ptr(),
+                                    out.data_ptr(), n_seqs, k, n_q_heads, n_kv_heads, head_dim,
+                                    C.c_void_p(stream.cuda_stream if stream is not None else 0))
+    if rc:
+        raise TidarError(rc, (lib.tidar_last_error(None) or b"").decode())
 
 
 def bf16_bits_to_f32(u16: np.ndarray) -> np.ndarray:

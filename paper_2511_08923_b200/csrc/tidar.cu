@@ -580,3 +580,72 @@ int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void
 }
 
 }  // extern "C"
+
+// =============================================================================
+// Attention without any allocation.
+//
+// Some hosts of this library may not allocate device memory at the moment they
+// need attention: a serving process whose memory pool has been handed over
+// completely to another component, a real-time loop that must not enter the
+// allocator (cudaMalloc can block on every other stream of the device), or a
+// plug-in that is given tensors but no allocator.  For them the per-row
+// visibility table that tidar_attention keeps in the context arena lives in the
+// fixed array below instead.  The array is part of the library image: every GPU
+// that loads the library carries it (TIDAR_STATIC_MAX_ROWS * 5 * 4 bytes) until
+// the process exits.
+// =============================================================================
+#define TIDAR_STATIC_MAX_ROWS 4352            /* 16 sequences of 16*17 slots */
+#define TIDAR_STATIC_MAX_DEVICES 64
+
+static __device__ __align__(256) int32_t g_static_rowmeta[5 * TIDAR_STATIC_MAX_ROWS];
+
+namespace {
+// Device address of g_static_rowmeta per device ordinal.  In host code the symbol's
+// name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress
+// with that device current.
+int32_t *g_static_ptr[TIDAR_STATIC_MAX_DEVICES] = {};
+}  // namespace
+
+extern "C" int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                                      int32_t pages_per_seq, const int32_t *seq_len, const void *k_local, const void *v_local,
+                                      void *out, int32_t n_seqs, int32_t k, int32_t n_q_heads, int32_t n_kv_heads,
+                                      int32_t head_dim, void *cuda_stream) {
+  if (!q || !k_pages || !v_pages || !page_table || !seq_len || !k_local || !v_local || !out)
+    return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: null argument");
+  if (head_dim != 64 && head_dim != 128) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: head_dim must be 64 or 128");
+  if (n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads)
+    return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: n_q_heads must be a positive multiple of n_kv_heads");
+  if (k < 1 || k > 32 || n_seqs < 1 || pages_per_seq < 1) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: bad k, n_seqs or pages_per_seq");
+  const long long rows = (long long)n_seqs * k * (k + 1);
+  if (rows > TIDAR_STATIC_MAX_ROWS)
+    return fail(nullptr, TIDAR_ECAPACITY, "tidar_attention_static: %lld rows exceed the built-in table of %d rows; use tidar_attention",
+                rows, TIDAR_STATIC_MAX_ROWS);
+  int dev = -1;
+  CUDA_TRY(nullptr, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= TIDAR_STATIC_MAX_DEVICES) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: device ordinal %d not supported", dev);
+  if (!g_static_ptr[dev]) {                    // first call on this device: resolve the table's device address
+    int32_t *p = nullptr;
+    CUDA_TRY(nullptr, cudaGetSymbolAddress((void **)&p, g_static_rowmeta));
+    if (!p) return fail(nullptr, TIDAR_ECUDA, "tidar_attention_static: no device address for the built-in table");
+    g_static_ptr[dev] = p;
+  }
+  int32_t *base = g_static_ptr[dev];
+  const int R = (int)rows;
+  RowMeta m{};
+  m.seq = base; m.pos = base + TIDAR_STATIC_MAX_ROWS; m.nvis = base + 2 * TIDAR_STATIC_MAX_ROWS;
+  m.loc0 = base + 3 * TIDAR_STATIC_MAX_ROWS; m.nloc = base + 4 * TIDAR_STATIC_MAX_ROWS;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  // every entry a row reads is rewritten here for rows [0, R): nothing has to start at zero
+  attn_meta_kernel<<<(R + 127) / 128, 128, 0, st>>>(m, seq_len, k, R);
+  KvGeom g{n_kv_heads, head_dim, 64, pages_per_seq, page_table};
+  const float scale = 1.0f / sqrtf((float)head_dim);
+  dim3 grid(R, n_q_heads);
+  if (head_dim == 128)
+    attn_replay_kernel<128><<<grid, 32, 0, st>>>((const bf16 *)q, (const bf16 *)k_pages, (const bf16 *)v_pages, g, m, (const bf16 *)k_local,
+                                                 (const bf16 *)v_local, (bf16 *)out, n_q_heads, scale);
+  else
+    attn_replay_kernel<64><<<grid, 32, 0, st>>>((const bf16 *)q, (const bf16 *)k_pages, (const bf16 *)v_pages, g, m, (const bf16 *)k_local,
+                                                (const bf16 *)v_local, (bf16 *)out, n_q_heads, scale);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  return TIDAR_OK;
+}
