@@ -382,7 +382,7 @@ def main():
         dist.destroy_process_group()
 
 
-DEFAULT_IMPL = 1
+DEFAULT_IMPL = 0
 # dram bytes per step of the projection kernels from an ncu capture (see profiles/); None until captured
 TRAFFIC_NOTE = {}
 

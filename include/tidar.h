@@ -180,6 +180,22 @@ int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const vo
                     const void *k_local, const void *v_local, void *out,
                     int32_t n_seqs, int32_t k);
 
+/* ---- one projection alone (microbenchmark and unit parity) ----------------------------
+ * out[r][n] = sum_k A[r][k] * W[n][k]: the weight-streaming small-M GEMM every projection
+ * of a step uses (QKV, O, gate/up, down, LM head; the step's k(k+1) token slots share one
+ * pass over the weights: paper Section 1, "free token slots").
+ *   A [R][K] bf16, W [N][K] bf16, out [R][N] fp32, all DEVICE, row-major, 16-byte aligned;
+ *   K a multiple of 64.  splits: K splits (1..8), 0 = the library's own choice; partial
+ *   sums are combined in a fixed order, so the result is deterministic.
+ * Enqueued on the context's stream; does not synchronise (see tidar_sync).
+ * Errors: EINVAL, ECAPACITY (R*N*splits exceeds the context's scratch), ECUDA.          */
+int tidar_gemm(tidar_ctx *ctx, const void *A, const void *W, int32_t R, int32_t N, int32_t K,
+               int32_t splits, float *out);
+
+/* Wait for everything enqueued on the context's stream and report a device-side
+ * timeout (TIDAR_EDEVICE_TIMEOUT) if a kernel's bounded wait gave up.                  */
+int tidar_sync(tidar_ctx *ctx);
+
 /* ---- structured-mask attention for callers that cannot allocate ---------------------
  * (The paper has no counterpart: this is a packaging variant of tidar_attention.)
  * Same computation, same tensor layouts and same mask as tidar_attention, but it needs

@@ -78,6 +78,8 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_debug_set_timing": (C.c_int, [ctxp, I32]),
         "tidar_debug_get_timing": (C.c_int, [ctxp, P(C.c_float)]),
         "tidar_attention": (C.c_int, [ctxp, VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32]),
+        "tidar_gemm": (C.c_int, [ctxp, VP, VP, I32, I32, I32, I32, VP]),
+        "tidar_sync": (C.c_int, [ctxp]),
         "tidar_attention_static": (C.c_int, [VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
     }
     for name, (res, args) in sig.items():
@@ -253,6 +255,15 @@ class Tidar:
         ms = (C.c_float * len(TC_NAMES))()
         self._check(self.lib.tidar_debug_get_timing(self.ctx, ms))
         return {n: float(ms[i]) for i, n in enumerate(TC_NAMES)}
+
+    def gemm(self, A, W, out, splits: int = 0):
+        """out[R][N] (fp32) = A[R][K] @ W[N][K]^T on caller-owned device tensors (see tidar.h)."""
+        R, K = A.shape
+        N = W.shape[0]
+        self._check(self.lib.tidar_gemm(self.ctx, A.data_ptr(), W.data_ptr(), R, N, K, splits, out.data_ptr()))
+
+    def sync(self):
+        self._check(self.lib.tidar_sync(self.ctx))
 
     def attention(self, q, k_pages, v_pages, page_table, seq_len, k_local, v_local, out, n_seqs: int, k: int):
         """Structured-mask attention alone, on caller-owned device tensors (see tidar.h)."""

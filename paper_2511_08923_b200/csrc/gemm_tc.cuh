@@ -1,0 +1,289 @@
+// Small-M weight-streaming GEMM on tcgen05 tensor cores.
+//
+//   out[r][n] = sum_k A[r][k] * W[n][k]      A [R][K] bf16 (activations, few rows),
+//                                            W [N][K] bf16 (weights, streamed once)
+//
+// A decode step has only k*(k+1) token slots per sequence (paper Section 3.3 footnote),
+// so every projection is a GEMM with a small row count and a weight matrix that is read
+// exactly once: the "free token slots" regime of the paper (Section 1; figure "Latency
+// Scaling").  The kernel therefore puts the WEIGHT rows on the 128 TMEM lanes (the MMA M
+// dimension) and the activation rows on the MMA N dimension (up to 288 = two instructions
+// of up to 144 columns), so no tensor-core work is wasted on padding rows.
+//
+// Work item = (row block, 128-row weight tile, K split).  Persistent CTAs, one per SM,
+// loop over items.  Warp roles: warp 0 issues TMA loads into a ring of shared-memory
+// stages, warp 1 issues the MMAs into one fp32 accumulator in TMEM, warps 2..9 drain the
+// accumulator into registers (which frees it for the next item at once) and then run the
+// epilogue from registers while the next item's MMAs proceed.
+#pragma once
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gemm_tc {
+
+constexpr int TILE_N = 128;         // weight rows per tile (TMEM lanes)
+constexpr int TILE_K = 64;          // bf16 elements per 128-byte swizzled row
+constexpr int MAX_ROWS = 288;       // activation rows per row block (2 x 144 TMEM columns)
+constexpr int THREADS = 320;
+constexpr int EPI_WARPS = 8;
+constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
+constexpr int SMEM_BUDGET = 220 * 1024;
+constexpr int TMEM_COLS = 512;
+
+enum Mode { MODE_SLAB = 0, MODE_SWIGLU = 1, MODE_ARGMAX = 2 };
+
+struct Args {
+  int R, N, K;              // activation rows in use, output features, input features
+  int rb_rows;              // rows per row block: multiple of 16, 16..288
+  int n_rb;                 // row blocks
+  int n_tiles;              // ceil(N / 128)
+  int S;                    // K splits
+  int kb_total;             // K / 64
+  int stages;               // shared-memory ring depth
+  int box_rows, n_box;      // activation rows per TMA box, boxes per stage
+  int n1, n2;               // MMA N of the two instructions (n2 may be 0)
+  // MODE_SLAB: fp32 out[split][r][n]
+  float *out; long long slab_stride; int ldo;
+  // MODE_SWIGLU: weight rows interleave (gate f, up f); H[r][f] = silu(gate) * up, bf16
+  bf16 *H; int ldh;
+  // MODE_ARGMAX: per (tile, lane quadrant) candidates, [n_tiles*4][R]; optional fp32 dump [R][ld_dump]
+  float *cand_val; int32_t *cand_idx; float *dump; int ld_dump; int col0;
+  int *status;              // device word set to 1 when a bounded wait gave up
+};
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
+
+template <int MODE>
+__global__ void __launch_bounds__(THREADS, 1)
+kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], tmem_full_bar, tmem_empty_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int a_stage_bytes = g.rb_rows * TILE_K * 2;
+  const int stage_bytes = W_STAGE_BYTES + a_stage_bytes;            // multiple of 1024 (rb_rows % 16 == 0)
+  const int n_items = g.n_rb * g.n_tiles * g.S;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < g.stages; ++s) { sm100::mbar_init(sm100::smem_u32(&full_bar[s]), 1); sm100::mbar_init(sm100::smem_u32(&empty_bar[s]), 1); }
+    sm100::mbar_init(sm100::smem_u32(&tmem_full_bar), 1);
+    sm100::mbar_init(sm100::smem_u32(&tmem_empty_bar), EPI_WARPS);
+    sm100::fence_mbar_init();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    sm100::tmem_alloc(sm100::smem_u32(&tmem_base_slot), TMEM_COLS);
+    sm100::tmem_relinquish();
+  }
+  sm100::tc_fence_before();
+  __syncthreads();
+  sm100::tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_slot;
+  volatile int *abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      sm100::prefetch_tensormap(&tmW);
+      sm100::prefetch_tensormap(&tmA);
+      const uint64_t pol_w = sm100::policy_evict_first(), pol_a = sm100::policy_evict_last();
+      int s = 0; uint32_t ph = 0; bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int split = item % g.S, tile = (item / g.S) % g.n_tiles, rb = item / (g.S * g.n_tiles);
+        const int kb0 = (int)((long long)g.kb_total * split / g.S), kb1 = (int)((long long)g.kb_total * (split + 1) / g.S);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!sm100::mbar_wait(sm100::smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) { ok = false; break; }
+          const uint32_t fb = sm100::smem_u32(&full_bar[s]);
+          const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
+          sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
+          sm100::tma_load_2d(sw, &tmW, fb, kb * TILE_K, tile * TILE_N, pol_w);
+          for (int b = 0; b < g.n_box; ++b)
+            sm100::tma_load_2d(sa + (uint32_t)(b * g.box_rows * TILE_K * 2), &tmA, fb, kb * TILE_K, rb * g.rb_rows + b * g.box_rows, pol_a);
+          if (++s == g.stages) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      const uint32_t idesc1 = sm100::make_idesc_bf16(TILE_N, g.n1), idesc2 = sm100::make_idesc_bf16(TILE_N, g.n2 ? g.n2 : 16);
+      int s = 0; uint32_t ph = 0; bool ok = true; uint32_t it = 0;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+        const int split = item % g.S;
+        const int kb0 = (int)((long long)g.kb_total * split / g.S), kb1 = (int)((long long)g.kb_total * (split + 1) / g.S);
+        if (!sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp)) { ok = false; break; }
+        sm100::tc_fence_after();
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!sm100::mbar_wait(sm100::smem_u32(&full_bar[s]), ph, abortp)) { ok = false; break; }
+          sm100::tc_fence_after();
+          const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < TILE_K / 16; ++kk) {
+            const uint32_t acc = (kb > kb0 || kk > 0) ? 1u : 0u;
+            const uint64_t wd = sm100::make_desc_sw128(sw + kk * 32);
+            sm100::mma_bf16_ss(tmem_acc, wd, sm100::make_desc_sw128(sa + kk * 32), idesc1, acc);
+            if (g.n2) sm100::mma_bf16_ss(tmem_acc + (uint32_t)g.n1, wd, sm100::make_desc_sw128(sa + (uint32_t)g.n1 * 128 + kk * 32), idesc2, acc);
+          }
+          sm100::mma_commit(sm100::smem_u32(&empty_bar[s]));     // stage reusable once these MMAs have read it
+          if (++s == g.stages) { s = 0; ph ^= 1u; }
+        }
+        if (ok) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
+      }
+    }
+  } else {
+    // ===================== epilogue =====================
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;
+    const int hc = ((g.rb_rows / 2 + 15) / 16) * 16;
+    const int c_begin = half ? hc : 0;
+    const int c_end = half ? g.rb_rows : (hc < g.rb_rows ? hc : g.rb_rows);
+    const int ncols = c_end - c_begin;           // multiple of 16, <= 144
+    uint32_t it = 0; bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+      const int split = item % g.S, tile = (item / g.S) % g.n_tiles, rb = item / (g.S * g.n_tiles);
+      if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
+      sm100::tc_fence_after();
+      uint32_t v[9][16];
+      const uint32_t t0 = tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin;
+#pragma unroll
+      for (int i = 0; i < 9; ++i)
+        if (i * 16 < ncols) sm100::tmem_ld16(t0 + i * 16, v[i]);
+      sm100::tmem_wait_ld();
+      sm100::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&tmem_empty_bar));   // accumulator free for the next item
+
+      const int n = tile * TILE_N + q * 32 + lane;       // this thread's output feature
+      const int r_base = rb * g.rb_rows + c_begin;
+      if (MODE == MODE_SLAB) {
+        float *o = g.out + (long long)split * g.slab_stride + n;
+        const bool n_ok = n < g.N;
+#pragma unroll
+        for (int i = 0; i < 9; ++i) {
+          if (i * 16 < ncols) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int r = r_base + i * 16 + j;
+              if (n_ok && r < g.R) o[(long long)r * g.ldo] = __uint_as_float(v[i][j]);
+            }
+          }
+        }
+      } else if (MODE == MODE_SWIGLU) {
+        // lane pairs (2j, 2j+1) hold gate and up of feature n/2; the even lane finishes
+        // column c, the odd lane column c+1, after one exchange per column pair.
+        const int f = n >> 1;
+        const bool f_ok = n < g.N;
+        const bool odd = lane & 1;
+#pragma unroll
+        for (int i = 0; i < 9; ++i) {
+          if (i * 16 < ncols) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+              const uint32_t send = odd ? v[i][j] : v[i][j + 1];
+              const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+              const float gate = __uint_as_float(odd ? recv : v[i][j]);
+              const float up = __uint_as_float(odd ? v[i][j + 1] : recv);
+              const int r = r_base + i * 16 + j + (odd ? 1 : 0);
+              if (f_ok && r < g.R) g.H[(long long)r * g.ldh + f] = __float2bfloat16(silu_mul(gate, up));
+            }
+          }
+        }
+      } else {
+        // per column: best (value, index) over the 32 features of this warp; lowest index
+        // wins ties, NaN never wins.
+        const bool n_ok = n < g.N;
+        const int cand_row = tile * 4 + q;
+#pragma unroll
+        for (int i = 0; i < 9; ++i) {
+          if (i * 16 < ncols) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int r = r_base + i * 16 + j;
+              float val = __uint_as_float(v[i][j]);
+              if (g.dump && n_ok && r < g.R) g.dump[(long long)r * g.ld_dump + n] = val;
+              int idx = g.col0 + n;
+              if (!n_ok || !(val == val)) { val = -INFINITY; idx = 0x7fffffff; }
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, val, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+              }
+              if (lane == 0 && r < g.R) {
+                g.cand_val[(long long)cand_row * g.R + r] = val;
+                g.cand_idx[(long long)cand_row * g.R + r] = idx == 0x7fffffff ? -1 : idx;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  sm100::tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    if (threadIdx.x == 0 && g.status) atomicExch(g.status, 1);
+    // give copies and MMAs that are still in flight time to land before the CTA's
+    // shared and tensor memory are released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    sm100::tc_fence_after();
+    sm100::tmem_dealloc(tmem_acc, TMEM_COLS);
+  }
+}
+
+// ---- host side ----------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns, 128-byte swizzle,
+// out-of-range elements read as zero.
+inline CUresult encode_2d(EncodeTiledFn fn, CUtensorMap *tm, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TILE_K, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+// Row-block geometry for R activation rows.
+inline void plan_rows(int R, Args &a) {
+  a.n_rb = (R + MAX_ROWS - 1) / MAX_ROWS;
+  const int per = (R + a.n_rb - 1) / a.n_rb;
+  a.rb_rows = (per + 15) / 16 * 16;
+  if (a.rb_rows <= 256) { a.box_rows = a.rb_rows; a.n_box = 1; a.n1 = a.rb_rows; a.n2 = 0; }
+  else { a.box_rows = a.rb_rows / 2; a.n_box = 2; a.n1 = ((a.rb_rows / 2 + 15) / 16) * 16; a.n2 = a.rb_rows - a.n1; }
+  const int stage = W_STAGE_BYTES + a.rb_rows * TILE_K * 2;
+  a.stages = SMEM_BUDGET / stage;
+  if (a.stages > 8) a.stages = 8;
+}
+inline size_t smem_bytes(const Args &a) { return (size_t)a.stages * (W_STAGE_BYTES + a.rb_rows * TILE_K * 2) + 1024; }
+
+// K splits: fill the SMs with whole waves of equally sized items, keeping at least
+// min_kb K blocks per item.
+inline int plan_splits(int n_items_unsplit, int kb_total, int n_sms, int max_splits, int min_kb) {
+  int best = 1; double best_eff = 0.0;
+  for (int s = 1; s <= max_splits; ++s) {
+    if (s > 1 && kb_total / s < min_kb) break;
+    const long long items = (long long)n_items_unsplit * s;
+    const long long waves = (items + n_sms - 1) / n_sms;
+    // time ~ waves * (k blocks per item + fixed per-item cost in k-block units)
+    const double per_item = (double)((kb_total + s - 1) / s) + 3.0;
+    const double eff = ((double)n_items_unsplit * kb_total) / ((double)waves * n_sms * per_item);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = s; }
+  }
+  return best;
+}
+
+}  // namespace gemm_tc

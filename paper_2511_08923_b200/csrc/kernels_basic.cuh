@@ -202,19 +202,41 @@ __global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int nco
   }
 }
 
-// Final argmax over per-CTA partial results [G][R] produced by the fused LM-head
-// epilogue: one thread per row scans the G candidates in order.
+// Final argmax over the candidates [G][R] produced by the fused LM-head epilogue (one
+// candidate per 32 vocabulary ids): one block per row; a candidate index of -1 means
+// "nothing valid".  Lowest index wins ties, which makes the result independent of the
+// order in which candidates are combined.
 __global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t *__restrict__ pi, int G, int R,
                                     float *__restrict__ best_val, int32_t *__restrict__ best_idx) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= R) return;
+  const int r = blockIdx.x;
   float bv = -INFINITY; int bi = 0x7fffffff;
-  for (int g = 0; g < G; ++g) {
+  for (int g = threadIdx.x; g < G; g += blockDim.x) {
     const float v = pv[(size_t)g * R + r]; const int i = pi[(size_t)g * R + r];
     if (i >= 0 && (v > bv || (v == bv && i < bi))) { bv = v; bi = i; }
   }
-  if (bi == 0x7fffffff) bi = 0;
-  best_val[r] = bv; best_idx[r] = bi;
+  __shared__ float sv[32]; __shared__ int si[32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o); const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+      if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
+    if (bi == 0x7fffffff) bi = 0;
+    best_val[r] = bv; best_idx[r] = bi;
+  }
+}
+
+// out[i] = sum over S slabs (fixed order) of in[s * stride + i].
+__global__ void slab_sum_kernel(const float *__restrict__ in, int S, size_t stride, size_t n, float *__restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float v = 0.f;
+  for (int s = 0; s < S; ++s) v += in[s * stride + i];
+  out[i] = v;
 }
 
 // ---------------------------------------------------------------------------

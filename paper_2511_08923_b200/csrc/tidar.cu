@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "kernels_basic.cuh"
 #include "kernels_replay.cuh"
+#include "gemm_tc.cuh"
 
 namespace {
 
@@ -38,6 +39,7 @@ struct tidar_ctx {
   int R_cap = 0, T_max = 0, pages_per_seq = 0, n_pages = 0, n_qkv = 0, S_max = 4, lm_chunk = 0;
   size_t pool_stride = 0;    // elements in one layer's K (or V) pool
   size_t partial_stride = 0; // elements between split-K partial slabs
+  size_t partials_cap = 0;   // floats in `partials`
   // arena carve-out (device)
   bf16 *kv = nullptr;
   RowMeta meta{};
@@ -56,6 +58,16 @@ struct tidar_ctx {
   // last pass
   int last_rows = 0, last_first_pos = 0;
   std::vector<int> pending_seqs; std::vector<int> pending_forced; bool pending = false;
+  // tensor-core path
+  gemm_tc::EncodeTiledFn encode = nullptr;
+  std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
+  CUtensorMap tm_lm;
+  struct AMap { const void *p; int rows, cols, box; CUtensorMap tm; };
+  std::vector<AMap> amaps;
+  int n_sms = 0;
+  int32_t *d_status = nullptr, *cand_idx = nullptr;
+  float *cand_val = nullptr;
+  int32_t *h_status = nullptr;
   // timing
   bool timing = false; std::vector<TimedLaunch> timed; float class_ms[TIDAR_TC_COUNT] = {};
   int cur_class = 0;
@@ -102,7 +114,7 @@ int validate(const tidar_config &c, std::string &why) {
   if (c.mask_token_id < 0 || c.mask_token_id >= c.vocab) return bad("mask_token_id out of range");
   if (c.beta != 1.0f) return bad("only beta = 1 is implemented");
   if (c.temperature != 0.0f) return bad("only greedy decoding (temperature 0) is implemented");
-  if (c.impl != 1) return bad("impl must be 1 (replay kernels); the tensor-core path is not built into this library yet");
+  if (c.impl != 0 && c.impl != 1) return bad("impl must be 0 (tensor-core kernels) or 1 (replay kernels)");
   if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return bad("rms_eps > 0 and rope_theta > 1 required");
   return TIDAR_OK;
 }
@@ -116,6 +128,7 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.n_qkv = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
   x.pool_stride = (size_t)x.n_pages * c.n_kv_heads * c.page_size * c.head_dim;
   x.lm_chunk = std::min(c.vocab, 16384);
+  x.S_max = c.impl == 0 ? 8 : 4;
   const size_t R = x.R_cap;
   const size_t widest = std::max<size_t>({(size_t)x.S_max * x.n_qkv, (size_t)x.S_max * c.d_model, (size_t)2 * c.d_ffn,
                                           (size_t)x.lm_chunk});
@@ -133,8 +146,14 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.d_out = cv.take<int32_t>((size_t)c.max_batch * (c.k_max + 1));
   x.d_prompt = cv.take<int32_t>(c.max_seq_len);
   x.d_arg_idx = cv.take<int32_t>(R); x.d_arg_val = cv.take<float>(R);
+  x.d_status = cv.take<int32_t>(64);
+  {
+    const size_t G = (size_t)((c.vocab + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N) * 4;
+    x.cand_val = cv.take<float>(G * R); x.cand_idx = cv.take<int32_t>(G * R);
+  }
   x.X = cv.take<float>(R * c.d_model);
   x.partials = cv.take<float>(R * widest);
+  x.partials_cap = R * widest;
   x.rope_cos = cv.take<float>(R * (c.head_dim / 2)); x.rope_sin = cv.take<float>(R * (c.head_dim / 2));
   x.A = cv.take<bf16>(R * c.d_model);
   x.Q = cv.take<bf16>(R * c.n_q_heads * c.head_dim);
@@ -178,13 +197,62 @@ KvGeom geom(const tidar_ctx *c) {
 }
 
 // ---- projections --------------------------------------------------------------
+// Tensor map of an activation matrix [rows][cols] (bf16) with a box of `box` rows; cached.
+const CUtensorMap *act_map(tidar_ctx *c, const void *p, int rows, int cols, int box) {
+  for (auto &m : c->amaps) if (m.p == p && m.rows == rows && m.cols == cols && m.box == box) return &m.tm;
+  tidar_ctx::AMap m{p, rows, cols, box, {}};
+  if (gemm_tc::encode_2d(c->encode, &m.tm, p, (uint64_t)rows, (uint64_t)cols, (uint32_t)box) != CUDA_SUCCESS) return nullptr;
+  if (c->amaps.size() > 256) c->amaps.erase(c->amaps.begin());
+  c->amaps.push_back(m);
+  return &c->amaps.back().tm;
+}
+
+// Tensor-core projection.  A [a_rows][K] (first R rows used), W described by tmW ([N][K]).
+//   MODE_SLAB  : S split-K partial slabs of fp32 [R][N] into c->partials (S chosen here)
+//   MODE_SWIGLU: bf16 c->H [R][N/2]
+//   MODE_ARGMAX: candidates for argmax_merge_kernel (+ optional logits dump)
+int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUtensorMap &tmW, int R, int N, int K, int cls,
+                   int *S_out, size_t *stride_out, float *slab_out = nullptr, int force_S = 0) {
+  gemm_tc::Args a{};
+  a.R = R; a.N = N; a.K = K;
+  gemm_tc::plan_rows(R, a);
+  a.n_tiles = (N + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N;
+  a.kb_total = K / gemm_tc::TILE_K;
+  a.S = 1;
+  if (mode == gemm_tc::MODE_SLAB) {
+    a.S = force_S > 0 ? std::min(force_S, a.kb_total) : gemm_tc::plan_splits(a.n_rb * a.n_tiles, a.kb_total, c->n_sms, c->S_max, 4);
+    a.out = slab_out ? slab_out : c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
+  } else if (mode == gemm_tc::MODE_SWIGLU) {
+    a.H = c->H; a.ldh = N / 2;
+  } else {
+    a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.dump = c->dbg_logits; a.ld_dump = c->cfg.vocab; a.col0 = 0;
+  }
+  a.status = c->d_status;
+  const CUtensorMap *tmA = act_map(c, A, a_rows, K, a.box_rows);
+  if (!tmA) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for an activation matrix (%d x %d, box %d)", a_rows, K, a.box_rows);
+  const int items = a.n_rb * a.n_tiles * a.S;
+  const int grid = std::min(items, c->n_sms);
+  const size_t smem = gemm_tc::smem_bytes(a);
+  Launch l(c, cls);
+  if (mode == gemm_tc::MODE_SLAB) gemm_tc::kernel<gemm_tc::MODE_SLAB><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  else if (mode == gemm_tc::MODE_SWIGLU) gemm_tc::kernel<gemm_tc::MODE_SWIGLU><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  else gemm_tc::kernel<gemm_tc::MODE_ARGMAX><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  if (S_out) *S_out = a.S;
+  if (stride_out) *stride_out = (size_t)R * N;
+  return TIDAR_OK;
+}
+
+enum Proj { P_QKV, P_O, P_GU, P_DOWN };
+
 // out = A[R][K] * W[N][K]^T as S split-K partial slabs of fp32 [R][N] (replay: S = 1).
-void gemm_partials(tidar_ctx *c, const bf16 *A, const bf16 *W, int R, int N, int K, float *out, int *S_out,
-                   size_t *stride_out, int cls) {
+int gemm_partials(tidar_ctx *c, const bf16 *A, int a_rows, const bf16 *W, const CUtensorMap *tmW, int R, int N, int K, float *out,
+                  int *S_out, size_t *stride_out, int cls) {
+  if (c->cfg.impl == 0) return gemm_tc_launch(c, gemm_tc::MODE_SLAB, A, a_rows, *tmW, R, N, K, cls, S_out, stride_out);
   Launch l(c, cls);
   dim3 grid((N + 63) / 64, (R + 63) / 64);
   gemm_replay_kernel<<<grid, 256, 0, c->stream>>>(A, K, W, K, out, N, R, N, K);
   *S_out = 1; *stride_out = (size_t)R * N;
+  return TIDAR_OK;
 }
 
 void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *Vp, const KvGeom &g, const bf16 *Kl,
@@ -216,42 +284,99 @@ int forward_rows(tidar_ctx *c, int R, bool with_head) {
     rope_table_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
   }
   int S = 0; size_t stride = 0;          // pending partials of the previous down projection
+  const bool tc = cf.impl == 0;
+  const int RA = c->R_cap;               // allocated rows of the activation buffers
+  int rc;
   for (int l = 0; l < cf.n_layers; ++l) {
     bf16 *Kp = c->kv + (size_t)(2 * l) * c->pool_stride, *Vp = Kp + c->pool_stride;
     launch_norm(c, R, c->partials, S, stride, c->attn_norm[l]);
     if (c->dbg_hidden)
       CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)l * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
                                   cudaMemcpyDeviceToDevice, c->stream));
-    gemm_partials(c, c->A, c->wqkv[l], R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
       rope_kv_kernel<<<dim3(R, Hq + 2 * Hkv), hd / 2, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     launch_attention(c, c->Q, Kp, Vp, g, c->Kloc, c->Vloc, c->O, R);
-    gemm_partials(c, c->O, c->wo[l], R, d, Hq * hd, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    if ((rc = gemm_partials(c, c->O, RA, c->wo[l], tc ? &c->tm_wo[l] : nullptr, R, d, Hq * hd, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     launch_norm(c, R, c->partials, S, stride, c->ffn_norm[l]);
-    gemm_partials(c, c->A, c->wgu[l], R, 2 * cf.d_ffn, d, c->partials, &S, &stride, TIDAR_TC_GEMM);
-    {
+    if (tc) {
+      if ((rc = gemm_tc_launch(c, gemm_tc::MODE_SWIGLU, c->A, RA, c->tm_wgu[l], R, 2 * cf.d_ffn, d, TIDAR_TC_GEMM, nullptr, nullptr))) return rc;
+    } else {
+      if ((rc = gemm_partials(c, c->A, RA, c->wgu[l], nullptr, R, 2 * cf.d_ffn, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
       Launch ll(c, TIDAR_TC_GEMM);
       const size_t n = (size_t)R * cf.d_ffn;
       swiglu_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->partials, R, cf.d_ffn, c->H);
     }
-    gemm_partials(c, c->H, c->wdown[l], R, d, cf.d_ffn, c->partials, &S, &stride, TIDAR_TC_GEMM);
+    if ((rc = gemm_partials(c, c->H, RA, c->wdown[l], tc ? &c->tm_wdown[l] : nullptr, R, d, cf.d_ffn, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
   }
   launch_norm(c, R, c->partials, S, stride, c->final_norm);
   if (c->dbg_hidden)
     CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)cf.n_layers * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
                                 cudaMemcpyDeviceToDevice, c->stream));
-  if (with_head) {
+  if (with_head && tc) {
+    if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
+    Launch ll(c, TIDAR_TC_LMHEAD);
+    const int G = ((cf.vocab + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N) * 4;
+    argmax_merge_kernel<<<R, 256, 0, c->stream>>>(c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
+  } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
-      gemm_partials(c, c->A, c->lm_head + (size_t)v0 * d, R, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD);
+      if ((rc = gemm_partials(c, c->A, RA, c->lm_head + (size_t)v0 * d, nullptr, R, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD))) return rc;
       Launch ll(c, TIDAR_TC_LMHEAD);
       argmax_chunk_kernel<<<R, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab);
     }
   }
   CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
+// Driver entry point for tensor-map encoding (resolved through the runtime so that the
+// library has no link-time dependency on the driver), tensor maps of every weight
+// matrix, kernel attributes.
+int init_tensor_core_path(tidar_ctx *c) {
+  const tidar_config &cf = c->cfg;
+  int dev = 0;
+  CUDA_TRY(c, cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CUDA_TRY(c, cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(c, TIDAR_ECUDA, "the tensor-core path needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
+  c->n_sms = prop.multiProcessorCount;
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CUDA_TRY(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
+  c->encode = (gemm_tc::EncodeTiledFn)fn;
+  const int d = cf.d_model, qo = cf.n_q_heads * cf.head_dim;
+  auto enc = [&](CUtensorMap *tm, const void *p, int rows, int cols) {
+    return gemm_tc::encode_2d(c->encode, tm, p, (uint64_t)rows, (uint64_t)cols, gemm_tc::TILE_N) == CUDA_SUCCESS;
+  };
+  c->tm_wqkv.resize(cf.n_layers); c->tm_wo.resize(cf.n_layers); c->tm_wgu.resize(cf.n_layers); c->tm_wdown.resize(cf.n_layers);
+  bool ok = enc(&c->tm_lm, c->lm_head, cf.vocab, d);
+  for (int l = 0; l < cf.n_layers && ok; ++l)
+    ok = enc(&c->tm_wqkv[l], c->wqkv[l], c->n_qkv, d) && enc(&c->tm_wo[l], c->wo[l], d, qo) &&
+         enc(&c->tm_wgu[l], c->wgu[l], 2 * cf.d_ffn, d) && enc(&c->tm_wdown[l], c->wdown[l], d, cf.d_ffn);
+  if (!ok) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix (pointers must be 16-byte aligned)");
+  const int max_smem = gemm_tc::SMEM_BUDGET + 1024;
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SLAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  return TIDAR_OK;
+}
+
+// Reads the device status word (already copied to pinned memory by the caller's
+// synchronised copy) and turns a device-side timeout into an error code.
+int check_device_status(tidar_ctx *c) {
+  if (c->cfg.impl != 0) return TIDAR_OK;
+  int st = 0;
+  CUDA_TRY(c, cudaMemcpyAsync(&st, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (st) {
+    cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
+    return fail(c, TIDAR_EDEVICE_TIMEOUT, "a bounded device-side wait gave up (status %d); results of this call are invalid", st);
+  }
   return TIDAR_OK;
 }
 
@@ -315,6 +440,7 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
                                                                        (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
   }
   CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaGetLastError());
   c->pending_seqs.assign(seqs, seqs + n_seqs);
   c->pending = true;
@@ -328,6 +454,8 @@ int finish_step(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
   c->pending = false;
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   if (c->timing) collect_timing(c);
+  if (c->h_status[0]) { c->h_status[0] = 0; cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
+    return fail(c, TIDAR_EDEVICE_TIMEOUT, "a bounded device-side wait gave up during the step; its results are invalid"); }
   const int km = c->cfg.k_max;
   for (size_t i = 0; i < c->pending_seqs.size(); ++i) {
     const int L = c->h_pinned[i * (km + 1)];
@@ -377,16 +505,22 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
     c->wo.push_back((const bf16 *)w->wo[l]); c->ffn_norm.push_back((const bf16 *)w->ffn_norm[l]);
     c->wgu.push_back((const bf16 *)w->w_gate_up[l]); c->wdown.push_back((const bf16 *)w->w_down[l]);
   }
+  if (cfg->impl == 0) {
+    if (int rc = init_tensor_core_path(c)) { std::string m = c->err; delete c; return fail(nullptr, rc, "%s", m.c_str()); }
+  }
   c->seqs.resize(cfg->max_batch);
   // free list in a scrambled order so that page tables are never contiguous
   c->free_pages.resize(c->n_pages);
   for (int i = 0; i < c->n_pages; ++i) c->free_pages[i] = i;
   uint32_t st = 0x9e3779b9u;
   for (int i = c->n_pages - 1; i > 0; --i) { st = st * 1664525u + 1013904223u; std::swap(c->free_pages[i], c->free_pages[(st >> 8) % (i + 1)]); }
-  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
+  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch + 16) * sizeof(int), cudaHostAllocDefault);
   if (e != cudaSuccess) { delete c; return fail(nullptr, TIDAR_ECUDA, "cudaHostAlloc: %s", cudaGetErrorString(e)); }
   c->h_stage = c->h_pinned + (size_t)cfg->max_batch * (cfg->k_max + 1);
+  c->h_status = c->h_stage + 2 * cfg->max_batch;
+  c->h_status[0] = 0;
   e = cudaMemsetAsync(c->d_seq_len, 0, cfg->max_batch * sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 64 * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_page_table, 0, (size_t)cfg->max_batch * c->pages_per_seq * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return fail(nullptr, TIDAR_ECUDA, "arena set-up: %s", cudaGetErrorString(e)); }
@@ -433,6 +567,7 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   CUDA_TRY(c, cudaGetLastError());
   if (c->timing) collect_timing(c);
+  if (int rc = check_device_status(c)) return rc;
   s.n = n_prompt; s.active = true;
   if (out_first) *out_first = c->h_pinned[0];
   return TIDAR_OK;
@@ -558,6 +693,39 @@ int tidar_debug_get_timing(tidar_ctx *c, float *ms) {
   if (!c || !ms) return TIDAR_EINVAL;
   for (int i = 0; i < TIDAR_TC_COUNT; ++i) ms[i] = c->class_ms[i];
   return TIDAR_OK;
+}
+
+int tidar_gemm(tidar_ctx *c, const void *A, const void *W, int32_t R, int32_t N, int32_t K, int32_t splits, float *out) {
+  if (!c) return TIDAR_EINVAL;
+  if (!A || !W || !out) return fail(c, TIDAR_EINVAL, "null argument");
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (R < 1 || N < 1 || K < 64 || K % 64) return fail(c, TIDAR_EINVAL, "R, N >= 1 and K a positive multiple of 64 required");
+  if (((uintptr_t)A | (uintptr_t)W) % 16) return fail(c, TIDAR_EINVAL, "A and W must be 16-byte aligned");
+  if (splits < 0 || splits > c->S_max) return fail(c, TIDAR_EINVAL, "splits must be in [0, %d]", c->S_max);
+  const size_t need = (size_t)(splits > 0 ? splits : c->S_max) * R * N;
+  if (need > c->partials_cap) return fail(c, TIDAR_ECAPACITY, "R*N*splits = %zu floats exceed the context's scratch (%zu)", need, c->partials_cap);
+  int S = 1; size_t stride = 0;
+  if (c->cfg.impl == 0) {
+    CUtensorMap tmW;
+    if (gemm_tc::encode_2d(c->encode, &tmW, W, (uint64_t)N, (uint64_t)K, gemm_tc::TILE_N) != CUDA_SUCCESS)
+      return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for W");
+    if (int rc = gemm_tc_launch(c, gemm_tc::MODE_SLAB, (const bf16 *)A, R, tmW, R, N, K, TIDAR_TC_GEMM, &S, &stride, nullptr, splits)) return rc;
+  } else {
+    if (int rc = gemm_partials(c, (const bf16 *)A, R, (const bf16 *)W, nullptr, R, N, K, c->partials, &S, &stride, TIDAR_TC_GEMM)) return rc;
+  }
+  {
+    Launch l(c, TIDAR_TC_GEMM);
+    const size_t n = (size_t)R * N;
+    slab_sum_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->partials, S, stride, n, out);
+  }
+  CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
+int tidar_sync(tidar_ctx *c) {
+  if (!c) return TIDAR_EINVAL;
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return check_device_status(c);
 }
 
 int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,

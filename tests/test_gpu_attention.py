@@ -11,7 +11,7 @@ from tidar_synth import CONFIGS, gen_normal_bf16, tensor_id
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [1]
+IMPLS = [0, 1]
 TOL = 3e-2          # unit-variance bf16 inputs; bf16 output rounding alone is ~1e-2 at |x| ~ 3
 
 

@@ -10,7 +10,7 @@ from tests.helpers import MARGIN, TOL_LOGITS, make_model, oracle_cfg, prompt_ids
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [1]
+IMPLS = [0, 1]
 
 
 def _gpu(sh, wt, impl, k_max=None, debug=1, max_batch=1, max_seq_len=512):
