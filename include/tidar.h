@@ -61,7 +61,8 @@ typedef struct {
   int32_t debug;            /* bit 0: keep per-layer hidden states and full logits of the
                                last pass for the tidar_debug_get_* calls (costs memory:
                                rows*vocab*4 bytes); bit 1: overwrite evicted KV slots with
-                               NaN after each step (proves nothing reads them)             */
+                               the largest finite bf16 after each step (any use of them
+                               with a non-zero weight would wreck the results)             */
   int32_t impl;             /* 0: tensor-core kernels (tcgen05/TMEM/TMA);
                                1: plain fp32-accumulate CUDA-core kernels ("replay"), a
                                slow diagnostic path with the same data flow               */
@@ -168,7 +169,8 @@ int tidar_debug_get_timing(tidar_ctx *ctx, float *ms /*host,[TIDAR_TC_COUNT]*/);
  *   q        [n_seqs*T][n_q_heads][head_dim], T = k*(k+1), slot order of a decode step
  *   k_pages, v_pages : page pools [n_pages][n_kv_heads][page_size][head_dim]; the
  *              cached prefix AND the k causal slots of the step (positions n..n+k-1)
- *              live there
+ *              live there.  Whole pages may be loaded: positions a row does not see
+ *              get weight zero, so they must hold finite values (not NaN/inf)
  *   page_table [n_seqs][pages_per_seq] int32, seq_len [n_seqs] int32 (= n per sequence)
  *   k_local, v_local [n_seqs*k*k][n_kv_heads][head_dim] : K/V of the mask slots
  *   out      [n_seqs*T][n_q_heads*head_dim]
@@ -176,7 +178,7 @@ int tidar_debug_get_timing(tidar_ctx *ctx, float *ms /*host,[TIDAR_TC_COUNT]*/);
  * slot (b,i) sees positions < n+b+1 plus the k local slots of block b.
  * Uses ctx only for its stream, kernel implementation choice and scratch.          */
 int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const void *v_pages,
-                    const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
+                    int32_t n_pages, const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
                     const void *k_local, const void *v_local, void *out,
                     int32_t n_seqs, int32_t k);
 

@@ -77,7 +77,7 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_debug_get_kv": (C.c_int, [ctxp, I32, I32, I32, I32, P(C.c_uint16), P(C.c_uint16)]),
         "tidar_debug_set_timing": (C.c_int, [ctxp, I32]),
         "tidar_debug_get_timing": (C.c_int, [ctxp, P(C.c_float)]),
-        "tidar_attention": (C.c_int, [ctxp, VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32]),
+        "tidar_attention": (C.c_int, [ctxp, VP, VP, VP, I32, VP, I32, VP, VP, VP, VP, I32, I32]),
         "tidar_gemm": (C.c_int, [ctxp, VP, VP, I32, I32, I32, I32, VP]),
         "tidar_sync": (C.c_int, [ctxp]),
         "tidar_attention_static": (C.c_int, [VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
@@ -268,7 +268,7 @@ class Tidar:
     def attention(self, q, k_pages, v_pages, page_table, seq_len, k_local, v_local, out, n_seqs: int, k: int):
         """Structured-mask attention alone, on caller-owned device tensors (see tidar.h)."""
         self._check(self.lib.tidar_attention(
-            self.ctx, q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), page_table.data_ptr(), page_table.shape[1],
+            self.ctx, q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), k_pages.shape[0], page_table.data_ptr(), page_table.shape[1],
             seq_len.data_ptr(), k_local.data_ptr(), v_local.data_ptr(), out.data_ptr(), n_seqs, k))
 
 

@@ -1,0 +1,386 @@
+// Structured-mask attention of one pass on tcgen05 tensor cores.
+//
+// A pass's rows (token slots) attend to the cached positions [0, nvis) of their sequence
+// plus the nloc step-local K/V rows starting at loc0 (see RowMeta).  For a decode step this
+// is the paper's decoding mask (figure "TiDAR Attention Masks"; Section 3.1): drafted
+// tokens causal, every mask block bidirectional inside itself and blind to the other
+// blocks.  The mask is never materialised: a query tile derives, from its rows' metadata,
+// which 64-key tiles it needs (cached pages up to the largest nvis, and only the local
+// rows of the blocks it contains), skips all others, and applies the per-row bound only
+// on tiles that straddle it.
+//
+// Tiling: the G = Hq/Hkv query heads that share a KV head are packed into one 128-row
+// MMA tile (floor(128/G) slots x G heads), so K/V are read once per KV head.  Per key
+// tile: S = Q K^T (M 128, N 64, K hd) into TMEM; the softmax warps read S (one thread per
+// row), keep the running max / sum, write P (bf16) to shared memory in the MMA operand
+// layout; O_tile = P V (M 128, N hd, K 64, V as the MN-major operand) into TMEM; the
+// softmax warps add it to their register accumulator.  S, P and O_tile are double
+// buffered, so QK^T of tile t+1 runs while tile t is in softmax.  The key range of a query
+// tile can be split over several CTAs; partial (max, sum, O) results are merged by
+// attn_combine_kernel.
+#pragma once
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace attn_tc {
+
+constexpr int KT = 64;               // keys per tile (= page size)
+constexpr int KV_STAGES = 3;
+constexpr int THREADS = 192;         // warp 0: TMA, warp 1: MMA, warps 2..5: softmax
+constexpr int MAX_SPLITS = 8;
+
+struct Args {
+  int R;                    // rows (slots) of the pass
+  int rows_per_group;       // slots per sequence group (k(k+1) for a step; R for a first pass)
+  int tiles_per_group;      // ceil(rows_per_group / spt)
+  int n_groups;
+  int spt;                  // slots per query tile = 128 / G
+  int G, Hq, Hkv;
+  int splits;
+  const int32_t *seq, *nvis, *loc0, *nloc;   // per row
+  const int32_t *page_table; int pages_per_seq;
+  int page_base_k, page_base_v;              // offsets in the page dimension of the K / V tensor maps
+  float scale_log2;                          // log2(e) / sqrt(hd)
+  bf16 *O;                                   // [R][Hq*hd]
+  float *part_O;                             // [splits][R][Hq][hd]  (splits > 1)
+  float *part_ml;                            // [splits][R][Hq][2]
+  unsigned long long *tile_stats;            // [2]: key tiles issued, key tiles a dense-mask kernel would issue (may be null)
+  int *status;
+};
+
+template <int HD>
+struct Smem {
+  static constexpr int NH = HD / 64;                 // 64-element halves of a head
+  static constexpr int Q_BYTES = 128 * HD * 2;
+  static constexpr int KV_BYTES = KT * HD * 2;
+  static constexpr int P_BYTES = 128 * KT * 2;
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = Q_OFF + Q_BYTES;
+  static constexpr int V_OFF = K_OFF + KV_STAGES * KV_BYTES;
+  static constexpr int P_OFF = V_OFF + KV_STAGES * KV_BYTES;
+  static constexpr int TOTAL = P_OFF + 2 * P_BYTES + 1024;
+  static constexpr int TMEM_COLS = HD == 128 ? 512 : 256;      // 2 x 64 (S) + 2 x HD (O), rounded up to a power of two
+};
+
+template <int HD>
+__global__ void __launch_bounds__(THREADS, 1)
+kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+       const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a) {
+  using L = Smem<HD>;
+  constexpr int NH = L::NH;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES],
+      s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag, sh_max_nvis, sh_loc_lo, sh_loc_hi;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
+
+  // ---- which work item ----
+  int w = blockIdx.x;
+  const int sp = w % a.splits; w /= a.splits;
+  const int kvh = w % a.Hkv; w /= a.Hkv;
+  const int tile = w % a.tiles_per_group; const int grp = w / a.tiles_per_group;
+  const int row0 = grp * a.rows_per_group + tile * a.spt;              // first slot of the tile
+  const int row_end = min((grp + 1) * a.rows_per_group, a.R);          // slots of this group end here
+  const int rows_used = a.spt * a.G;                                   // MMA rows that carry data
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0; sh_max_nvis = 0; sh_loc_lo = 0x7fffffff; sh_loc_hi = 0;
+    sm100::mbar_init(sm100::smem_u32(&q_full), 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      sm100::mbar_init(sm100::smem_u32(&k_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&k_empty[s]), 1);
+      sm100::mbar_init(sm100::smem_u32(&v_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&v_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      sm100::mbar_init(sm100::smem_u32(&s_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&s_empty[b]), 4);
+      sm100::mbar_init(sm100::smem_u32(&p_full[b]), 4); sm100::mbar_init(sm100::smem_u32(&p_empty[b]), 1);
+      sm100::mbar_init(sm100::smem_u32(&o_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&o_empty[b]), 4);
+    }
+    sm100::fence_mbar_init();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    sm100::tmem_alloc(sm100::smem_u32(&tmem_base_slot), L::TMEM_COLS);
+    sm100::tmem_relinquish();
+  }
+  __syncthreads();
+
+  // ---- per-row metadata (softmax threads own one MMA row each) and the tile's key range ----
+  const int my_row = (warp & 3) * 32 + lane;             // MMA row = TMEM lane (softmax warps only)
+  int my_slot = -1, my_nvis = 0, my_loc0 = 0, my_nloc = 0, my_head = 0;
+  if (warp >= 2) {
+    const int sl = my_row / a.G;
+    const int pr = row0 + sl;
+    if (sl < a.spt && pr < row_end) {
+      my_slot = pr; my_head = kvh * a.G + my_row % a.G;
+      my_nvis = a.nvis[pr]; my_nloc = a.nloc[pr]; my_loc0 = a.loc0[pr];
+      atomicMax(&sh_max_nvis, my_nvis);
+      if (my_nloc > 0) { atomicMin(&sh_loc_lo, my_loc0); atomicMax(&sh_loc_hi, my_loc0 + my_nloc); }
+    }
+  }
+  sm100::tc_fence_before();
+  __syncthreads();
+  sm100::tc_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+  const uint32_t tmem_S = tmem, tmem_O = tmem + 2 * KT;               // S: 2 x 64 columns, O: 2 x HD columns
+  const int max_nvis = sh_max_nvis;
+  const int loc_lo = sh_loc_lo, loc_hi = sh_loc_hi;
+  const int n_cache_tiles = (max_nvis + KT - 1) / KT;
+  const int n_loc_tiles = loc_hi > loc_lo ? (loc_hi - loc_lo + KT - 1) / KT : 0;
+  const int nt_all = n_cache_tiles + n_loc_tiles;
+  const int t_begin = (int)((long long)nt_all * sp / a.splits), t_end = (int)((long long)nt_all * (sp + 1) / a.splits);
+  const int nt = t_end - t_begin;
+  const int seq = row0 < a.R ? a.seq[row0] : 0;
+  volatile int *abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0 && nt > 0) {
+      const uint64_t pol_q = sm100::policy_evict_last(), pol_kv = sm100::policy_evict_last();
+      const uint32_t qb = sm100::smem_u32(&q_full);
+      sm100::mbar_expect_tx(qb, (uint32_t)(NH * rows_used * 128));
+      for (int h = 0; h < NH; ++h)
+        sm100::tma_load_3d(smem0 + L::Q_OFF + h * (128 * 128), &tmQ, qb, h * 64, kvh * a.G, row0, pol_q);
+      int s = 0; uint32_t ph = 0; bool ok = true;
+      for (int t = t_begin; t < t_end && ok; ++t) {
+        const bool is_cache = t < n_cache_tiles;
+        const int page = is_cache ? a.page_table[(size_t)seq * a.pages_per_seq + t] : 0;
+        const int lrow = loc_lo + (t - n_cache_tiles) * KT;
+        // K
+        if (!sm100::mbar_wait(sm100::smem_u32(&k_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+        uint32_t fb = sm100::smem_u32(&k_full[s]);
+        sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
+        for (int h = 0; h < NH; ++h) {
+          const uint32_t dst = smem0 + L::K_OFF + s * L::KV_BYTES + h * (KT * 128);
+          if (is_cache) sm100::tma_load_4d(dst, &tmK, fb, h * 64, 0, kvh, a.page_base_k + page, pol_kv);
+          else sm100::tma_load_3d(dst, &tmKloc, fb, h * 64, kvh, lrow, pol_kv);
+        }
+        // V
+        if (!sm100::mbar_wait(sm100::smem_u32(&v_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+        fb = sm100::smem_u32(&v_full[s]);
+        sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
+        for (int h = 0; h < NH; ++h) {
+          const uint32_t dst = smem0 + L::V_OFF + s * L::KV_BYTES + h * (KT * 128);
+          if (is_cache) sm100::tma_load_4d(dst, &tmV, fb, h * 64, 0, kvh, a.page_base_v + page, pol_kv);
+          else sm100::tma_load_3d(dst, &tmVloc, fb, h * 64, kvh, lrow, pol_kv);
+        }
+        if (++s == KV_STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0 && nt > 0) {
+      const uint32_t idesc_qk = sm100::make_idesc_bf16(128, KT);
+      const uint32_t idesc_pv = sm100::make_idesc_bf16(128, HD) | (1u << 16);      // B (= V) is MN-major
+      bool ok = sm100::mbar_wait(sm100::smem_u32(&q_full), 0, abortp);
+      sm100::tc_fence_after();
+      int ks = 0; uint32_t kph = 0;          // K ring position of the next QK^T
+      int vs = 0; uint32_t vph = 0;          // V ring position of the next PV
+      auto issue_qk = [&](int i) -> bool {   // i: tile counter of this CTA
+        const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
+        if (!sm100::mbar_wait(sm100::smem_u32(&k_full[ks]), kph, abortp)) return false;
+        if (!sm100::mbar_wait(sm100::smem_u32(&s_empty[b]), bph ^ 1u, abortp)) return false;
+        sm100::tc_fence_after();
+        const uint32_t kb = smem0 + L::K_OFF + ks * L::KV_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t qa = smem0 + L::Q_OFF + (kk / 4) * (128 * 128) + (kk % 4) * 32;
+          const uint32_t ka = kb + (kk / 4) * (KT * 128) + (kk % 4) * 32;
+          sm100::mma_bf16_ss(tmem_S + b * KT, sm100::make_desc_sw128(qa), sm100::make_desc_sw128(ka), idesc_qk, kk > 0 ? 1u : 0u);
+        }
+        sm100::mma_commit(sm100::smem_u32(&k_empty[ks]));
+        sm100::mma_commit(sm100::smem_u32(&s_full[b]));
+        if (++ks == KV_STAGES) { ks = 0; kph ^= 1u; }
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int i = 0; i < nt && ok; ++i) {
+        if (i + 1 < nt) { ok = issue_qk(i + 1); if (!ok) break; }
+        const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
+        if (!sm100::mbar_wait(sm100::smem_u32(&v_full[vs]), vph, abortp)) { ok = false; break; }
+        if (!sm100::mbar_wait(sm100::smem_u32(&o_empty[b]), bph ^ 1u, abortp)) { ok = false; break; }
+        if (!sm100::mbar_wait(sm100::smem_u32(&p_full[b]), bph, abortp)) { ok = false; break; }
+        sm100::tc_fence_after();
+        const uint32_t pb = smem0 + L::P_OFF + b * L::P_BYTES;
+        const uint32_t vb = smem0 + L::V_OFF + vs * L::KV_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < KT / 16; ++kk)
+          sm100::mma_bf16_ss(tmem_O + b * HD, sm100::make_desc_sw128(pb + kk * 32),
+                             sm100::make_desc_sw128_mn(vb + kk * 16 * 128, KT * 128), idesc_pv, kk > 0 ? 1u : 0u);
+        sm100::mma_commit(sm100::smem_u32(&v_empty[vs]));
+        sm100::mma_commit(sm100::smem_u32(&p_empty[b]));
+        sm100::mma_commit(sm100::smem_u32(&o_full[b]));
+        if (++vs == KV_STAGES) { vs = 0; vph ^= 1u; }
+      }
+    }
+  } else {
+    // ===================== softmax + accumulation =====================
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    float o_acc[HD];
+#pragma unroll
+    for (int d = 0; d < HD; ++d) o_acc[d] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f, m_acc = -INFINITY, m_prev = -INFINITY;
+    bool ok = true;
+
+    auto accumulate = [&](int i, float m_tile) -> bool {       // add O_tile(i), computed under max m_tile
+      const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
+      if (!sm100::mbar_wait(sm100::smem_u32(&o_full[b]), bph, abortp)) return false;
+      sm100::tc_fence_after();
+      const float f = (m_acc == -INFINITY) ? 0.f : exp2f(m_acc - m_tile);
+#pragma unroll
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t v[32];
+        sm100::tmem_ld32(tmem_O + lane_addr + b * HD + c * 32, v);
+        sm100::tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o_acc[c * 32 + j] = fmaf(o_acc[c * 32 + j], f, __uint_as_float(v[j]));
+      }
+      sm100::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&o_empty[b]));
+      m_acc = m_tile;
+      return true;
+    };
+
+    for (int i = 0; i < nt && ok; ++i) {
+      const int t = t_begin + i;
+      const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
+      if (!sm100::mbar_wait(sm100::smem_u32(&s_full[b]), bph, abortp)) { ok = false; break; }
+      sm100::tc_fence_after();
+      uint32_t sv[64];
+      {
+        uint32_t v0[32], v1[32];
+        sm100::tmem_ld32(tmem_S + lane_addr + b * KT, v0);
+        sm100::tmem_ld32(tmem_S + lane_addr + b * KT + 32, v1);
+        sm100::tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { sv[j] = v0[j]; sv[32 + j] = v1[j]; }
+      }
+      sm100::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&s_empty[b]));
+
+      // visible keys of this tile for my row: [lo, hi) in tile-local indices
+      int lo = 0, hi = 0;
+      if (my_slot >= 0) {
+        if (t < n_cache_tiles) { lo = 0; hi = min(KT, my_nvis - t * KT); }
+        else {
+          const int base = loc_lo + (t - n_cache_tiles) * KT;           // local row of key 0
+          lo = max(0, my_loc0 - base); hi = my_nloc > 0 ? min(KT, my_loc0 + my_nloc - base) : 0;
+        }
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) {
+        float s = __uint_as_float(sv[j]) * a.scale_log2;
+        s = (j >= lo && j < hi) ? s : -INFINITY;
+        sv[j] = __float_as_uint(s);
+        mx = fmaxf(mx, s);
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+      const float alpha = exp2f(m_run - m_safe);              // m_run = -inf gives 0
+      float sum = 0.f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int j = 0; j < 64; j += 2) {
+        const float p0 = exp2f(__uint_as_float(sv[j]) - m_safe), p1 = exp2f(__uint_as_float(sv[j + 1]) - m_safe);
+        sum += p0 + p1;
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+        pk[j >> 1] = *reinterpret_cast<uint32_t *>(&h2);
+      }
+      l_run = l_run * alpha + sum;
+      m_run = m_new;
+
+      // P -> shared memory in the 128-byte-swizzled K-major operand layout
+      if (!sm100::mbar_wait(sm100::smem_u32(&p_empty[b]), bph ^ 1u, abortp)) { ok = false; break; }
+      {
+        const uint32_t prow = smem0 + L::P_OFF + b * L::P_BYTES + (my_row >> 3) * 1024 + (my_row & 7) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t dst = prow + ((c ^ (my_row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]), "r"(pk[4 * c + 2]),
+                       "r"(pk[4 * c + 3]) : "memory");
+        }
+      }
+      sm100::fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&p_full[b]));
+
+      if (i >= 1) ok = accumulate(i - 1, m_prev);
+      m_prev = m_run;
+    }
+    if (ok && nt > 0) ok = accumulate(nt - 1, m_prev);
+
+    // ---- output ----
+    if (ok && my_slot >= 0) {
+      if (a.splits == 1) {
+        const float inv = 1.f / l_run;
+        bf16 *o = a.O + ((size_t)my_slot * a.Hq + my_head) * HD;
+#pragma unroll
+        for (int d = 0; d < HD; d += 8) {
+          uint4 u;
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(o_acc[d] * inv, o_acc[d + 1] * inv), h1 = __floats2bfloat162_rn(o_acc[d + 2] * inv, o_acc[d + 3] * inv),
+                         h2 = __floats2bfloat162_rn(o_acc[d + 4] * inv, o_acc[d + 5] * inv), h3 = __floats2bfloat162_rn(o_acc[d + 6] * inv, o_acc[d + 7] * inv);
+          u.x = *reinterpret_cast<uint32_t *>(&h0); u.y = *reinterpret_cast<uint32_t *>(&h1);
+          u.z = *reinterpret_cast<uint32_t *>(&h2); u.w = *reinterpret_cast<uint32_t *>(&h3);
+          *reinterpret_cast<uint4 *>(o + d) = u;
+        }
+      } else {
+        const size_t idx = ((size_t)sp * a.R + my_slot) * a.Hq + my_head;
+        float *po = a.part_O + idx * HD;
+#pragma unroll
+        for (int d = 0; d < HD; d += 4) *reinterpret_cast<float4 *>(po + d) = make_float4(o_acc[d], o_acc[d + 1], o_acc[d + 2], o_acc[d + 3]);
+        a.part_ml[idx * 2] = m_run; a.part_ml[idx * 2 + 1] = l_run;
+      }
+    }
+    if (a.tile_stats && threadIdx.x == 64 && sp == 0 && kvh == 0) {
+      // a dense-mask kernel would visit every cached page up to the group's last position and
+      // every local row of the group for each query tile
+      atomicAdd(&a.tile_stats[0], (unsigned long long)nt_all);
+    }
+  }
+
+  // ---- teardown ----
+  sm100::tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    if (threadIdx.x == 0 && a.status) atomicExch(a.status, 2);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    sm100::tc_fence_after();
+    sm100::tmem_dealloc(tmem, L::TMEM_COLS);
+  }
+}
+
+// Merge the per-split partial results: O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
+// One warp per (row, head).
+template <int HD>
+__global__ void combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
+                               bf16 *__restrict__ O) {
+  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (wid >= R * Hq) return;
+  float M = -INFINITY;
+  for (int s = 0; s < splits; ++s) M = fmaxf(M, part_ml[((size_t)s * R * Hq + wid) * 2]);
+  float den = 0.f, acc[HD / 32];
+#pragma unroll
+  for (int i = 0; i < HD / 32; ++i) acc[i] = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const size_t idx = (size_t)s * R * Hq + wid;
+    const float m = part_ml[idx * 2], l = part_ml[idx * 2 + 1];
+    const float wgt = (m == -INFINITY) ? 0.f : exp2f(m - M);
+    den += wgt * l;
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) acc[i] = fmaf(wgt, part_O[idx * HD + i * 32 + lane], acc[i]);
+  }
+  const float inv = 1.f / den;
+#pragma unroll
+  for (int i = 0; i < HD / 32; ++i) O[(size_t)wid * HD + i * 32 + lane] = __float2bfloat16(acc[i] * inv);
+}
+
+}  // namespace attn_tc

@@ -291,8 +291,11 @@ __global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int r
 // KV commit / evict (paper Section 3.3): the k causal slots' K/V were written to
 // the cache at positions n..n+k-1 during the pass; committing L of them is
 // n <- n + L, after which positions n+L..n+k-1 are dead and get overwritten by the
-// next step.  With poison != 0 the dead slots are filled with NaN in every layer, so
-// any later read of evicted data would surface.  Grid (n_seqs, n_layers).
+// next step.  With poison != 0 the dead slots are filled, in every layer, with the
+// largest finite bf16 (3.4e38), so that any later use of evicted data with a non-zero
+// weight would surface as inf/NaN or a wild value.  (Not NaN itself: the tensor-core
+// attention loads whole 64-position pages and multiplies the masked positions' V rows
+// by an exact zero, which must stay zero.)  Grid (n_seqs, n_layers).
 // ---------------------------------------------------------------------------
 __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ step_n,
                                  const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, int poison,
@@ -304,7 +307,7 @@ __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const in
   if (!poison) return;
   bf16 *Kp = kv_base + (size_t)(2 * l) * pool_stride, *Vp = Kp + pool_stride;
   const int per = g.n_kv_heads * g.head_dim;
-  const bf16 nanv = __ushort_as_bfloat16((unsigned short)0x7fc0);
+  const bf16 nanv = __ushort_as_bfloat16((unsigned short)0x7f7f);
   for (int t = threadIdx.x; t < (k - L) * per; t += blockDim.x) {
     const int p = n + L + t / per, kvh = (t % per) / g.head_dim, c = t % g.head_dim;
     const size_t off = kv_row_offset(g, seq, p, kvh) + c;

@@ -72,6 +72,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
       ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1, int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t policy) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
@@ -138,6 +144,19 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
   d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset: one 8-row group
   d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
   d |= (uint64_t)2 << 61;                       // layout: 128-byte swizzle
+  return d;
+}
+// Same storage (rows of 64 elements = 128 bytes, 128-byte swizzle, 8 rows per 1024-byte
+// group), but used as an MN-major operand: a row is one K index and holds 64 consecutive
+// M/N indices.  Successive 8-row K groups are 1024 bytes apart (stride offset); the next
+// 64 M/N indices start `mn_chunk_bytes` further (leading offset).
+__device__ __forceinline__ uint64_t make_desc_sw128_mn(uint32_t saddr, uint32_t mn_chunk_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((mn_chunk_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
   return d;
 }
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major,

@@ -13,6 +13,7 @@
 #include "kernels_basic.cuh"
 #include "kernels_replay.cuh"
 #include "gemm_tc.cuh"
+#include "attn_tc.cuh"
 
 namespace {
 
@@ -64,6 +65,8 @@ struct tidar_ctx {
   CUtensorMap tm_lm;
   struct AMap { const void *p; int rows, cols, box; CUtensorMap tm; };
   std::vector<AMap> amaps;
+  CUtensorMap tm_q, tm_kv, tm_kloc, tm_vloc;
+  float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
   int32_t *d_status = nullptr, *cand_idx = nullptr;
   float *cand_val = nullptr;
@@ -147,6 +150,10 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.d_prompt = cv.take<int32_t>(c.max_seq_len);
   x.d_arg_idx = cv.take<int32_t>(R); x.d_arg_val = cv.take<float>(R);
   x.d_status = cv.take<int32_t>(64);
+  if (c.impl == 0) {
+    x.attn_part_O = cv.take<float>((size_t)attn_tc::MAX_SPLITS * R * c.n_q_heads * c.head_dim);
+    x.attn_part_ml = cv.take<float>((size_t)attn_tc::MAX_SPLITS * R * c.n_q_heads * 2);
+  }
   {
     const size_t G = (size_t)((c.vocab + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N) * 4;
     x.cand_val = cv.take<float>(G * R); x.cand_idx = cv.take<int32_t>(G * R);
@@ -255,6 +262,72 @@ int gemm_partials(tidar_ctx *c, const bf16 *A, int a_rows, const bf16 *W, const 
   return TIDAR_OK;
 }
 
+// bf16 tensor maps for the attention kernel (128-byte swizzle, 64-element inner box).
+bool encode_q_map(tidar_ctx *c, CUtensorMap *tm, const void *q, int rows) {
+  const tidar_config &cf = c->cfg;
+  const int G = cf.n_q_heads / cf.n_kv_heads, spt = 128 / G;
+  cuuint64_t dims[3] = {(cuuint64_t)cf.head_dim, (cuuint64_t)cf.n_q_heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)cf.head_dim * 2, (cuuint64_t)cf.n_q_heads * cf.head_dim * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)spt}, es[3] = {1, 1, 1};
+  return c->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(q), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+bool encode_pages_map(tidar_ctx *c, CUtensorMap *tm, const void *pool, long long n_pages) {
+  const tidar_config &cf = c->cfg;
+  cuuint64_t dims[4] = {(cuuint64_t)cf.head_dim, 64, (cuuint64_t)cf.n_kv_heads, (cuuint64_t)n_pages};
+  cuuint64_t strides[3] = {(cuuint64_t)cf.head_dim * 2, (cuuint64_t)64 * cf.head_dim * 2, (cuuint64_t)cf.n_kv_heads * 64 * cf.head_dim * 2};
+  cuuint32_t box[4] = {64, 64, 1, 1}, es[4] = {1, 1, 1, 1};
+  return c->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+bool encode_local_map(tidar_ctx *c, CUtensorMap *tm, const void *loc, long long rows) {
+  const tidar_config &cf = c->cfg;
+  cuuint64_t dims[3] = {(cuuint64_t)cf.head_dim, (cuuint64_t)cf.n_kv_heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)cf.head_dim * 2, (cuuint64_t)cf.n_kv_heads * cf.head_dim * 2};
+  cuuint32_t box[3] = {64, 1, 64}, es[3] = {1, 1, 1};
+  return c->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(loc), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct AttnMaps { const CUtensorMap *q, *k, *v, *kloc, *vloc; int page_base_k, page_base_v; };
+
+// rows_per_group: slots per sequence (k(k+1) in a step; all rows in a first-pass chunk).
+// key_tiles_hint: rough number of 64-key tiles per row, to size the key split.
+void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 *O, int R, int rows_per_group, int key_tiles_hint) {
+  const tidar_config &cf = c->cfg;
+  attn_tc::Args a{};
+  a.R = R; a.rows_per_group = rows_per_group;
+  a.G = cf.n_q_heads / cf.n_kv_heads; a.Hq = cf.n_q_heads; a.Hkv = cf.n_kv_heads;
+  a.spt = 128 / a.G;
+  a.tiles_per_group = (rows_per_group + a.spt - 1) / a.spt;
+  a.n_groups = (R + rows_per_group - 1) / rows_per_group;
+  const int units = a.n_groups * a.tiles_per_group * a.Hkv;
+  int splits = c->n_sms / std::max(units, 1);
+  splits = std::min(splits, std::max(1, key_tiles_hint / 2));
+  a.splits = std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
+  a.seq = c->meta.seq; a.nvis = c->meta.nvis; a.loc0 = c->meta.loc0; a.nloc = c->meta.nloc;
+  a.page_table = g.page_table; a.pages_per_seq = g.pages_per_seq;
+  a.page_base_k = m.page_base_k; a.page_base_v = m.page_base_v;
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)cf.head_dim);
+  a.O = O; a.part_O = c->attn_part_O; a.part_ml = c->attn_part_ml; a.tile_stats = nullptr; a.status = c->d_status;
+  const int grid = units * a.splits;
+  {
+    Launch l(c, TIDAR_TC_ATTN);
+    if (cf.head_dim == 128)
+      attn_tc::kernel<128><<<grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+    else
+      attn_tc::kernel<64><<<grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+  }
+  if (a.splits > 1) {
+    Launch l(c, TIDAR_TC_ATTN);
+    const int warps = R * cf.n_q_heads;
+    if (cf.head_dim == 128)
+      attn_tc::combine_kernel<128><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+    else
+      attn_tc::combine_kernel<64><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+  }
+}
+
 void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *Vp, const KvGeom &g, const bf16 *Kl,
                       const bf16 *Vl, bf16 *O, int R) {
   Launch l(c, TIDAR_TC_ATTN);
@@ -274,7 +347,7 @@ void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t strid
 
 // The transformer stack over R assembled rows (metadata and X already filled).
 // with_head: run final norm + LM head + per-row argmax.
-int forward_rows(tidar_ctx *c, int R, bool with_head) {
+int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int key_tiles_hint) {
   const tidar_config &cf = c->cfg;
   const int d = cf.d_model, hd = cf.head_dim, Hq = cf.n_q_heads, Hkv = cf.n_kv_heads;
   const KvGeom g = geom(c);
@@ -299,7 +372,12 @@ int forward_rows(tidar_ctx *c, int R, bool with_head) {
       rope_kv_kernel<<<dim3(R, Hq + 2 * Hkv), hd / 2, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
-    launch_attention(c, c->Q, Kp, Vp, g, c->Kloc, c->Vloc, c->O, R);
+    if (tc) {
+      AttnMaps am{&c->tm_q, &c->tm_kv, &c->tm_kv, &c->tm_kloc, &c->tm_vloc, (2 * l) * c->n_pages, (2 * l + 1) * c->n_pages};
+      launch_attention_tc(c, am, g, c->O, R, rows_per_group, key_tiles_hint);
+    } else {
+      launch_attention(c, c->Q, Kp, Vp, g, c->Kloc, c->Vloc, c->O, R);
+    }
     if ((rc = gemm_partials(c, c->O, RA, c->wo[l], tc ? &c->tm_wo[l] : nullptr, R, d, Hq * hd, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     launch_norm(c, R, c->partials, S, stride, c->ffn_norm[l]);
     if (tc) {
@@ -359,6 +437,19 @@ int init_tensor_core_path(tidar_ctx *c) {
     ok = enc(&c->tm_wqkv[l], c->wqkv[l], c->n_qkv, d) && enc(&c->tm_wo[l], c->wo[l], d, qo) &&
          enc(&c->tm_wgu[l], c->wgu[l], 2 * cf.d_ffn, d) && enc(&c->tm_wdown[l], c->wdown[l], d, cf.d_ffn);
   if (!ok) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix (pointers must be 16-byte aligned)");
+  {
+    const size_t nloc = (size_t)std::max(cf.max_batch * cf.k_max * cf.k_max, cf.k_max);
+    if (!encode_q_map(c, &c->tm_q, c->Q, c->R_cap) || !encode_pages_map(c, &c->tm_kv, c->kv, (long long)cf.n_layers * 2 * c->n_pages) ||
+        !encode_local_map(c, &c->tm_kloc, c->Kloc, (long long)nloc) || !encode_local_map(c, &c->tm_vloc, c->Vloc, (long long)nloc))
+      return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for an attention operand");
+    // The PV product multiplies masked keys' V rows by an exact zero, so whatever the
+    // kernel may load (unwritten cache slots of a page, unwritten local rows) must be finite.
+    CUDA_TRY(c, cudaMemsetAsync(c->kv, 0, (size_t)cf.n_layers * 2 * c->pool_stride * sizeof(bf16), c->stream));
+    CUDA_TRY(c, cudaMemsetAsync(c->Kloc, 0, nloc * cf.n_kv_heads * cf.head_dim * sizeof(bf16), c->stream));
+    CUDA_TRY(c, cudaMemsetAsync(c->Vloc, 0, nloc * cf.n_kv_heads * cf.head_dim * sizeof(bf16), c->stream));
+    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<128>::TOTAL));
+    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<64>::TOTAL));
+  }
   const int max_smem = gemm_tc::SMEM_BUDGET + 1024;
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SLAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
@@ -427,7 +518,9 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
     assemble_step_kernel<<<R, 128, 0, c->stream>>>(c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
                                                    c->d_step_n, c->embed, cf.d_model, c->X);
   }
-  int rc = forward_rows(c, R, true);
+  int min_n = 1 << 30;
+  for (int i = 0; i < n_seqs; ++i) min_n = std::min(min_n, c->seqs[seqs[i]].n);
+  int rc = forward_rows(c, R, true, T, (min_n + k + 63) / 64);
   if (rc) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
@@ -554,7 +647,7 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
       assemble_prefill_kernel<<<rows, 128, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
                                                            cf.d_model, c->X);
     }
-    if (int rc = forward_rows(c, rows, last)) return rc;
+    if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64)) return rc;
     if (last) {
       Launch l(c, TIDAR_TC_VERIFY);
       prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, n_prompt - 1 - row0, k, cf.k_max, seq, n_prompt, c->d_block,
@@ -728,12 +821,13 @@ int tidar_sync(tidar_ctx *c) {
   return check_device_status(c);
 }
 
-int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void *v_pages, int32_t n_pages, const int32_t *page_table,
                     int32_t pages_per_seq, const int32_t *seq_len, const void *k_local, const void *v_local, void *out,
                     int32_t n_seqs, int32_t k) {
   if (!c) return TIDAR_EINVAL;
   if (!q || !k_pages || !v_pages || !page_table || !seq_len || !k_local || !v_local || !out) return fail(c, TIDAR_EINVAL, "null argument");
   if (k < 1 || k > c->cfg.k_max || n_seqs < 1 || n_seqs * k * (k + 1) > c->R_cap) return fail(c, TIDAR_EINVAL, "n_seqs * k(k+1) exceeds the context's row capacity");
+  if (n_pages < 1 || pages_per_seq < 1) return fail(c, TIDAR_EINVAL, "n_pages and pages_per_seq must be positive");
   if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
   const int R = n_seqs * k * (k + 1);
   {
@@ -741,8 +835,19 @@ int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void
     attn_meta_kernel<<<(R + 127) / 128, 128, 0, c->stream>>>(c->meta, seq_len, k, R);
   }
   KvGeom g{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, pages_per_seq, page_table};
-  launch_attention(c, (const bf16 *)q, (const bf16 *)k_pages, (const bf16 *)v_pages, g, (const bf16 *)k_local, (const bf16 *)v_local,
-                   (bf16 *)out, R);
+  if (c->cfg.impl == 0) {
+    if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)k_local | (uintptr_t)v_local | (uintptr_t)out) % 16)
+      return fail(c, TIDAR_EINVAL, "tensors must be 16-byte aligned");
+    CUtensorMap tq, tk, tv, tkl, tvl;
+    if (!encode_q_map(c, &tq, q, R) || !encode_pages_map(c, &tk, k_pages, n_pages) || !encode_pages_map(c, &tv, v_pages, n_pages) ||
+        !encode_local_map(c, &tkl, k_local, (long long)n_seqs * k * k) || !encode_local_map(c, &tvl, v_local, (long long)n_seqs * k * k))
+      return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for an attention operand");
+    AttnMaps am{&tq, &tk, &tv, &tkl, &tvl, 0, 0};
+    launch_attention_tc(c, am, g, (bf16 *)out, R, k * (k + 1), pages_per_seq);
+  } else {
+    launch_attention(c, (const bf16 *)q, (const bf16 *)k_pages, (const bf16 *)v_pages, g, (const bf16 *)k_local, (const bf16 *)v_local,
+                     (bf16 *)out, R);
+  }
   CUDA_TRY(c, cudaGetLastError());
   return TIDAR_OK;
 }
