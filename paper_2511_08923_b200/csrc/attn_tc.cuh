@@ -64,7 +64,7 @@ struct Smem {
 
 template <int HD>
 __global__ void __launch_bounds__(THREADS, 1)
-kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
        const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a) {
   using L = Smem<HD>;
   constexpr int NH = L::NH;
@@ -361,7 +361,7 @@ kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensor
 // Merge the per-split partial results: O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
 // One warp per (row, head).
 template <int HD>
-__global__ void combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
+__global__ void attn_combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
                                bf16 *__restrict__ O) {
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (wid >= R * Hq) return;

@@ -55,7 +55,7 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + 
 
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
-kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], tmem_full_bar, tmem_empty_bar;
   __shared__ uint32_t tmem_base_slot;

@@ -241,9 +241,9 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   const int grid = std::min(items, c->n_sms);
   const size_t smem = gemm_tc::smem_bytes(a);
   Launch l(c, cls);
-  if (mode == gemm_tc::MODE_SLAB) gemm_tc::kernel<gemm_tc::MODE_SLAB><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
-  else if (mode == gemm_tc::MODE_SWIGLU) gemm_tc::kernel<gemm_tc::MODE_SWIGLU><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
-  else gemm_tc::kernel<gemm_tc::MODE_ARGMAX><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  if (mode == gemm_tc::MODE_SLAB) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  else if (mode == gemm_tc::MODE_SWIGLU) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  else gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
   if (S_out) *S_out = a.S;
   if (stride_out) *stride_out = (size_t)R * N;
   return TIDAR_OK;
@@ -314,17 +314,17 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   {
     Launch l(c, TIDAR_TC_ATTN);
     if (cf.head_dim == 128)
-      attn_tc::kernel<128><<<grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      attn_tc::attn_tc_kernel<128><<<grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
     else
-      attn_tc::kernel<64><<<grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      attn_tc::attn_tc_kernel<64><<<grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
   }
   if (a.splits > 1) {
     Launch l(c, TIDAR_TC_ATTN);
     const int warps = R * cf.n_q_heads;
     if (cf.head_dim == 128)
-      attn_tc::combine_kernel<128><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      attn_tc::attn_combine_kernel<128><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
     else
-      attn_tc::combine_kernel<64><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      attn_tc::attn_combine_kernel<64><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
   }
 }
 
@@ -447,13 +447,13 @@ int init_tensor_core_path(tidar_ctx *c) {
     CUDA_TRY(c, cudaMemsetAsync(c->kv, 0, (size_t)cf.n_layers * 2 * c->pool_stride * sizeof(bf16), c->stream));
     CUDA_TRY(c, cudaMemsetAsync(c->Kloc, 0, nloc * cf.n_kv_heads * cf.head_dim * sizeof(bf16), c->stream));
     CUDA_TRY(c, cudaMemsetAsync(c->Vloc, 0, nloc * cf.n_kv_heads * cf.head_dim * sizeof(bf16), c->stream));
-    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<128>::TOTAL));
-    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<64>::TOTAL));
+    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<128>::TOTAL));
+    CUDA_TRY(c, cudaFuncSetAttribute(attn_tc::attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::Smem<64>::TOTAL));
   }
   const int max_smem = gemm_tc::SMEM_BUDGET + 1024;
-  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SLAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::kernel<gemm_tc::MODE_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
   return TIDAR_OK;
 }
 
