@@ -178,17 +178,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       sm100::tc_fence_after();
       int ks = 0; uint32_t kph = 0;          // K ring position of the next QK^T
       int vs = 0; uint32_t vph = 0;          // V ring position of the next PV
+      // descriptors are built once; the issue loop only adds 16-byte-unit offsets
+      const uint64_t q_desc = sm100::make_desc_sw128(smem0 + L::Q_OFF);
+      const uint64_t k_desc0 = sm100::make_desc_sw128(smem0 + L::K_OFF);
+      const uint64_t p_desc0 = sm100::make_desc_sw128(smem0 + L::P_OFF);
+      const uint64_t v_desc0 = sm100::make_desc_sw128_mn(smem0 + L::V_OFF, KT * 128);
+      constexpr uint64_t KV16 = L::KV_BYTES >> 4, P16 = L::P_BYTES >> 4;
       auto issue_qk = [&](int i) -> bool {   // i: tile counter of this CTA
         const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
         if (!sm100::mbar_wait(sm100::smem_u32(&k_full[ks]), kph, abortp)) return false;
         if (!sm100::mbar_wait(sm100::smem_u32(&s_empty[b]), bph ^ 1u, abortp)) return false;
         sm100::tc_fence_after();
-        const uint32_t kb = smem0 + L::K_OFF + ks * L::KV_BYTES;
+        const uint64_t kd = k_desc0 + (uint64_t)ks * KV16;
+        const uint32_t d = tmem_S + b * KT;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t qa = smem0 + L::Q_OFF + (kk / 4) * (128 * 128) + (kk % 4) * 32;
-          const uint32_t ka = kb + (kk / 4) * (KT * 128) + (kk % 4) * 32;
-          sm100::mma_bf16_ss(tmem_S + b * KT, sm100::make_desc_sw128(qa), sm100::make_desc_sw128(ka), idesc_qk, kk > 0 ? 1u : 0u);
+          // 64-element half kk/4 of the head: Q halves are 128 rows x 128 B apart, K halves 64 rows x 128 B
+          sm100::mma_bf16_ss(d, q_desc + (kk / 4) * (128 * 128 / 16) + (kk % 4) * 2, kd + (kk / 4) * (KT * 128 / 16) + (kk % 4) * 2, idesc_qk,
+                             kk > 0 ? 1u : 0u);
         }
         sm100::mma_commit(sm100::smem_u32(&k_empty[ks]));
         sm100::mma_commit(sm100::smem_u32(&s_full[b]));
@@ -203,12 +210,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (!sm100::mbar_wait(sm100::smem_u32(&o_empty[b]), bph ^ 1u, abortp)) { ok = false; break; }
         if (!sm100::mbar_wait(sm100::smem_u32(&p_full[b]), bph, abortp)) { ok = false; break; }
         sm100::tc_fence_after();
-        const uint32_t pb = smem0 + L::P_OFF + b * L::P_BYTES;
-        const uint32_t vb = smem0 + L::V_OFF + vs * L::KV_BYTES;
+        const uint64_t pd = p_desc0 + (uint64_t)b * P16;
+        const uint64_t vd = v_desc0 + (uint64_t)vs * KV16;
+        const uint32_t d = tmem_O + b * HD;
 #pragma unroll
-        for (int kk = 0; kk < KT / 16; ++kk)
-          sm100::mma_bf16_ss(tmem_O + b * HD, sm100::make_desc_sw128(pb + kk * 32),
-                             sm100::make_desc_sw128_mn(vb + kk * 16 * 128, KT * 128), idesc_pv, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per instruction: 32 B along a P row, 16 V rows (2048 B)
+          sm100::mma_bf16_ss(d, pd + kk * 2, vd + kk * (16 * 128 / 16), idesc_pv, kk > 0 ? 1u : 0u);
         sm100::mma_commit(sm100::smem_u32(&v_empty[vs]));
         sm100::mma_commit(sm100::smem_u32(&p_empty[b]));
         sm100::mma_commit(sm100::smem_u32(&o_full[b]));

@@ -46,7 +46,8 @@ struct Args {
   float *out; long long slab_stride; int ldo;
   // MODE_SWIGLU: weight rows interleave (gate f, up f); H[r][f] = silu(gate) * up, bf16
   bf16 *H; int ldh;
-  // MODE_ARGMAX: per (tile, lane quadrant) candidates, [n_tiles*4][R]; optional fp32 dump [R][ld_dump]
+  // MODE_ARGMAX: per (CTA, lane quadrant) candidates, [gridDim*4][R] (index -1 = none; the caller
+  // pre-fills the index table with -1); optional fp32 dump [R][ld_dump]
   float *cand_val; int32_t *cand_idx; float *dump; int ld_dump; int col0;
   int *status;              // device word set to 1 when a bounded wait gave up
 };
@@ -109,27 +110,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
+    // One thread issues every MMA, so its instruction count per K block bounds the whole
+    // kernel: descriptors are built once and advanced with plain adds (the start-address
+    // field counts 16-byte units and never carries out of its 14 bits inside shared memory).
     if (lane == 0) {
       const uint32_t idesc1 = sm100::make_idesc_bf16(TILE_N, g.n1), idesc2 = sm100::make_idesc_bf16(TILE_N, g.n2 ? g.n2 : 16);
+      const uint64_t desc0 = sm100::make_desc_sw128(smem0);             // stage 0 weights
+      const uint64_t stage16 = (uint64_t)(stage_bytes >> 4);
+      const uint64_t a_off16 = (uint64_t)(W_STAGE_BYTES >> 4), a2_off16 = (uint64_t)(g.n1 * 8);
+      const uint32_t tmem_acc2 = tmem_acc + (uint32_t)g.n1;
+      const bool two = g.n2 != 0;
       int s = 0; uint32_t ph = 0; bool ok = true; uint32_t it = 0;
+      uint64_t wd = desc0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
         const int split = item % g.S;
         const int kb0 = (int)((long long)g.kb_total * split / g.S), kb1 = (int)((long long)g.kb_total * (split + 1) / g.S);
         if (!sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp)) { ok = false; break; }
         sm100::tc_fence_after();
+        uint32_t acc = 0u;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!sm100::mbar_wait(sm100::smem_u32(&full_bar[s]), ph, abortp)) { ok = false; break; }
           sm100::tc_fence_after();
-          const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
+          const uint64_t ad = wd + a_off16;
+          if (two) {
+            const uint64_t ad2 = ad + a2_off16;
 #pragma unroll
-          for (int kk = 0; kk < TILE_K / 16; ++kk) {
-            const uint32_t acc = (kb > kb0 || kk > 0) ? 1u : 0u;
-            const uint64_t wd = sm100::make_desc_sw128(sw + kk * 32);
-            sm100::mma_bf16_ss(tmem_acc, wd, sm100::make_desc_sw128(sa + kk * 32), idesc1, acc);
-            if (g.n2) sm100::mma_bf16_ss(tmem_acc + (uint32_t)g.n1, wd, sm100::make_desc_sw128(sa + (uint32_t)g.n1 * 128 + kk * 32), idesc2, acc);
+            for (int kk = 0; kk < TILE_K / 16; ++kk) {
+              sm100::mma_bf16_ss(tmem_acc, wd + 2 * kk, ad + 2 * kk, idesc1, acc);
+              sm100::mma_bf16_ss(tmem_acc2, wd + 2 * kk, ad2 + 2 * kk, idesc2, acc);
+              acc = 1u;
+            }
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < TILE_K / 16; ++kk) {
+              sm100::mma_bf16_ss(tmem_acc, wd + 2 * kk, ad + 2 * kk, idesc1, acc);
+              acc = 1u;
+            }
           }
           sm100::mma_commit(sm100::smem_u32(&empty_bar[s]));     // stage reusable once these MMAs have read it
-          if (++s == g.stages) { s = 0; ph ^= 1u; }
+          wd += stage16;
+          if (++s == g.stages) { s = 0; ph ^= 1u; wd = desc0; }
         }
         if (ok) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
       }
@@ -143,6 +163,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int c_end = half ? g.rb_rows : (hc < g.rb_rows ? hc : g.rb_rows);
     const int ncols = c_end - c_begin;           // multiple of 16, <= 144
     uint32_t it = 0; bool ok = true;
+    // MODE_ARGMAX: running best of column c_begin + 32*slot + lane, and the row block it belongs to
+    float best_v[5]; int best_i[5]; int cur_rb = -1;
+#pragma unroll
+    for (int k = 0; k < 5; ++k) { best_v[k] = -INFINITY; best_i[k] = 0x7fffffff; }
+    auto flush_best = [&]() {
+      if (cur_rb < 0) return;
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        const int cidx = k * 32 + lane;
+        const int r = cur_rb * g.rb_rows + c_begin + cidx;
+        if (cidx < ncols && r < g.R) {
+          const long long o = (long long)(blockIdx.x * 4 + q) * g.R + r;
+          g.cand_val[o] = best_v[k]; g.cand_idx[o] = best_i[k] == 0x7fffffff ? -1 : best_i[k];
+        }
+        best_v[k] = -INFINITY; best_i[k] = 0x7fffffff;
+      }
+    };
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
       const int split = item % g.S, tile = (item / g.S) % g.n_tiles, rb = item / (g.S * g.n_tiles);
       if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
@@ -193,10 +230,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
         }
       } else {
-        // per column: best (value, index) over the 32 features of this warp; lowest index
-        // wins ties, NaN never wins.
+        // Per column: best (value, index) over the 32 features of this warp, folded into a
+        // running best over all tiles this CTA processes (column c is kept by lane c % 32).
+        // Lowest index wins ties, NaN never wins.
+        if (rb != cur_rb) { flush_best(); cur_rb = rb; }
         const bool n_ok = n < g.N;
-        const int cand_row = tile * 4 + q;
 #pragma unroll
         for (int i = 0; i < 9; ++i) {
           if (i * 16 < ncols) {
@@ -213,15 +251,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
                 if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
               }
-              if (lane == 0 && r < g.R) {
-                g.cand_val[(long long)cand_row * g.R + r] = val;
-                g.cand_idx[(long long)cand_row * g.R + r] = idx == 0x7fffffff ? -1 : idx;
+              const int cidx = i * 16 + j;
+              if (lane == (cidx & 31) && (val > best_v[cidx >> 5] || (val == best_v[cidx >> 5] && idx < best_i[cidx >> 5]))) {
+                best_v[cidx >> 5] = val; best_i[cidx >> 5] = idx;
               }
             }
           }
         }
       }
     }
+    if (MODE == MODE_ARGMAX) flush_best();
   }
 
   // ---- teardown ----

@@ -3,6 +3,17 @@
 #pragma once
 #include "common.cuh"
 
+// One embedding row (bf16, d a multiple of 8) -> fp32, 16-byte loads.
+__device__ __forceinline__ void embed_row_to_f32(const bf16 *__restrict__ e, float *__restrict__ x, int d) {
+  for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
+    const uint4 u = *reinterpret_cast<const uint4 *>(e + c);
+    const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&u);
+    const float2 a = __bfloat1622float2(p[0]), b = __bfloat1622float2(p[1]), cc = __bfloat1622float2(p[2]), dd = __bfloat1622float2(p[3]);
+    *reinterpret_cast<float4 *>(x + c) = make_float4(a.x, a.y, b.x, b.y);
+    *reinterpret_cast<float4 *>(x + c + 4) = make_float4(cc.x, cc.y, dd.x, dd.y);
+  }
+}
+
 // ---------------------------------------------------------------------------
 // Slot assembly + embedding gather for a decode step.
 // Slot layout per sequence (k causal slots, then k blocks of k mask slots;
@@ -36,8 +47,7 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
       m.cache_pos[r] = -1; m.local_idx[r] = s * k * k + b * k + i;
     }
   }
-  const bf16 *e = embed + (size_t)id * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) X[(size_t)r * d + c] = __bfloat162float(e[c]);
+  embed_row_to_f32(embed + (size_t)id * d, X + (size_t)r * d, d);
 }
 
 // Prefill chunk: rows g = row0 .. row0+rows-1 of [prompt ; k mask tokens]
@@ -57,8 +67,7 @@ __global__ void assemble_prefill_kernel(RowMeta m, int seq, int row0, int n_prom
       m.nvis[r] = n_prompt; m.loc0[r] = 0; m.nloc[r] = k; m.cache_pos[r] = -1; m.local_idx[r] = g - n_prompt;
     }
   }
-  const bf16 *e = embed + (size_t)id * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) X[(size_t)r * d + c] = __bfloat162float(e[c]);
+  embed_row_to_f32(embed + (size_t)id * d, X + (size_t)r * d, d);
 }
 
 // Row metadata for the stand-alone attention entry point (same slot layout as a step).
@@ -103,11 +112,15 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials,
   __shared__ float red[THREADS / 32];
   const int r = blockIdx.x;
   float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += THREADS) {
-    float v = X[(size_t)r * d + c];
-    for (int s = 0; s < S; ++s) v += partials[s * partial_stride + (size_t)r * d + c];
-    row[c] = v;
-    ss += v * v;
+  float *xr = X + (size_t)r * d;
+  for (int c = threadIdx.x * 4; c < d; c += THREADS * 4) {
+    float4 v = *reinterpret_cast<const float4 *>(xr + c);
+    for (int s = 0; s < S; ++s) {
+      const float4 p = *reinterpret_cast<const float4 *>(partials + s * partial_stride + (size_t)r * d + c);
+      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    }
+    *reinterpret_cast<float4 *>(row + c) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -116,10 +129,14 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials,
 #pragma unroll
   for (int i = 0; i < THREADS / 32; ++i) tot += red[i];
   const float inv = rsqrtf(tot / (float)d + eps);
-  for (int c = threadIdx.x; c < d; c += THREADS) {
-    const float v = row[c];
-    if (S > 0) X[(size_t)r * d + c] = v;
-    A[(size_t)r * d + c] = __float2bfloat16(v * inv * __bfloat162float(gain[c]));
+  for (int c = threadIdx.x * 4; c < d; c += THREADS * 4) {
+    const float4 v = *reinterpret_cast<const float4 *>(row + c);
+    if (S > 0) *reinterpret_cast<float4 *>(xr + c) = v;
+    const uint2 gb = *reinterpret_cast<const uint2 *>(gain + c);
+    const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gb.x)), g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gb.y));
+    __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * inv * g0.x, v.y * inv * g0.y), o1 = __floats2bfloat162_rn(v.z * inv * g1.x, v.w * inv * g1.y);
+    uint2 ob; ob.x = *reinterpret_cast<uint32_t *>(&o0); ob.y = *reinterpret_cast<uint32_t *>(&o1);
+    *reinterpret_cast<uint2 *>(A + (size_t)r * d + c) = ob;
   }
 }
 
@@ -128,37 +145,53 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials,
 // [S][R][(Hq+2Hkv)*hd].  Q heads are rotated and stored bf16 [R][Hq][hd]; K heads are
 // rotated, V heads copied; both go to the paged cache at the row's cache position
 // (causal slots: kept if accepted, evicted otherwise; paper Section 3.3) or to the
-// step-local scratch (mask slots, never cached).  Grid (R, Hq+2Hkv), hd/2 threads.
+// step-local scratch (mask slots, never cached).  One block per row.
 // ---------------------------------------------------------------------------
-__global__ void rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
-                               RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
-                               bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
-                               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
-  const int r = blockIdx.x, h = blockIdx.y, i = threadIdx.x, half = hd / 2;
-  const int N = (Hq + 2 * Hkv) * hd;
-  const size_t base = (size_t)r * N + (size_t)h * hd;
-  float x1 = 0.f, x2 = 0.f;
-  for (int s = 0; s < S; ++s) {
-    x1 += partials[s * partial_stride + base + i];
-    x2 += partials[s * partial_stride + base + i + half];
-  }
-  bf16 *dst;
-  if (h < Hq) {
-    dst = Q + ((size_t)r * Hq + h) * hd;
-  } else {
-    const bool isk = h < Hq + Hkv;
-    const int kvh = isk ? h - Hq : h - Hq - Hkv;
-    const int cp = m.cache_pos[r];
-    if (cp >= 0) dst = (isk ? Kpool : Vpool) + kv_row_offset(g, m.seq[r], cp, kvh);
-    else dst = (isk ? Kloc : Vloc) + ((size_t)m.local_idx[r] * Hkv + kvh) * hd;
-    if (!isk) {  // V: no rotation
-      dst[i] = __float2bfloat16(x1); dst[i + half] = __float2bfloat16(x2);
-      return;
+__global__ void __launch_bounds__(256)
+rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
+               RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
+               bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
+               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
+  // one block per row; a work unit is 4 consecutive dims i..i+3 of the first half of one
+  // head together with their rotation partners i+hd/2..
+  const int r = blockIdx.x, half = hd / 2, upr = half / 4;          // units per head
+  const int H = Hq + 2 * Hkv, N = H * hd;
+  const int cp = m.cache_pos[r], seq = m.seq[r], li = m.local_idx[r];
+  for (int u = threadIdx.x; u < H * upr; u += blockDim.x) {
+    const int h = u / upr, i = (u % upr) * 4;
+    const size_t base = (size_t)r * N + (size_t)h * hd + i;
+    float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;
+    for (int s = 0; s < S; ++s) {
+      const float4 a = *reinterpret_cast<const float4 *>(partials + s * partial_stride + base);
+      const float4 b = *reinterpret_cast<const float4 *>(partials + s * partial_stride + base + half);
+      x1.x += a.x; x1.y += a.y; x1.z += a.z; x1.w += a.w;
+      x2.x += b.x; x2.y += b.y; x2.z += b.z; x2.w += b.w;
     }
+    bf16 *dst;
+    bool rotate = true;
+    if (h < Hq) {
+      dst = Q + ((size_t)r * Hq + h) * hd;
+    } else {
+      const bool isk = h < Hq + Hkv;
+      const int kvh = isk ? h - Hq : h - Hq - Hkv;
+      if (cp >= 0) dst = (isk ? Kpool : Vpool) + kv_row_offset(g, seq, cp, kvh);
+      else dst = (isk ? Kloc : Vloc) + ((size_t)li * Hkv + kvh) * hd;
+      rotate = isk;
+    }
+    float4 y1 = x1, y2 = x2;
+    if (rotate) {
+      const float4 c = *reinterpret_cast<const float4 *>(cs + r * half + i), sv = *reinterpret_cast<const float4 *>(sn + r * half + i);
+      y1 = make_float4(x1.x * c.x - x2.x * sv.x, x1.y * c.y - x2.y * sv.y, x1.z * c.z - x2.z * sv.z, x1.w * c.w - x2.w * sv.w);
+      y2 = make_float4(x2.x * c.x + x1.x * sv.x, x2.y * c.y + x1.y * sv.y, x2.z * c.z + x1.z * sv.z, x2.w * c.w + x1.w * sv.w);
+    }
+    __nv_bfloat162 a0 = __floats2bfloat162_rn(y1.x, y1.y), a1 = __floats2bfloat162_rn(y1.z, y1.w);
+    __nv_bfloat162 b0 = __floats2bfloat162_rn(y2.x, y2.y), b1 = __floats2bfloat162_rn(y2.z, y2.w);
+    uint2 o1, o2;
+    o1.x = *reinterpret_cast<uint32_t *>(&a0); o1.y = *reinterpret_cast<uint32_t *>(&a1);
+    o2.x = *reinterpret_cast<uint32_t *>(&b0); o2.y = *reinterpret_cast<uint32_t *>(&b1);
+    *reinterpret_cast<uint2 *>(dst + i) = o1;
+    *reinterpret_cast<uint2 *>(dst + i + half) = o2;
   }
-  const float c = cs[r * half + i], s = sn[r * half + i];
-  dst[i] = __float2bfloat16(x1 * c - x2 * s);
-  dst[i + half] = __float2bfloat16(x2 * c + x1 * s);
 }
 
 // SwiGLU on an fp32 [R][2*ffn] projection whose columns interleave (gate_f, up_f).

@@ -155,7 +155,7 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
     x.attn_part_ml = cv.take<float>((size_t)attn_tc::MAX_SPLITS * R * c.n_q_heads * 2);
   }
   {
-    const size_t G = (size_t)((c.vocab + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N) * 4;
+    const size_t G = 4 * 256;            // (CTAs of the LM-head kernel <= SMs) x 4 lane quadrants
     x.cand_val = cv.take<float>(G * R); x.cand_idx = cv.take<int32_t>(G * R);
   }
   x.X = cv.take<float>(R * c.d_model);
@@ -342,7 +342,7 @@ void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *V
 void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t stride, const bf16 *gain) {
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
-  rmsnorm_reduce_kernel<256><<<R, 256, d * sizeof(float), c->stream>>>(c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+  rmsnorm_reduce_kernel<512><<<R, 512, d * sizeof(float), c->stream>>>(c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
 }
 
 // The transformer stack over R assembled rows (metadata and X already filled).
@@ -369,7 +369,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
-      rope_kv_kernel<<<dim3(R, Hq + 2 * Hkv), hd / 2, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+      rope_kv_kernel<<<R, 256, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     if (tc) {
@@ -395,9 +395,10 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)cf.n_layers * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
                                 cudaMemcpyDeviceToDevice, c->stream));
   if (with_head && tc) {
+    const int G = c->n_sms * 4;          // upper bound of (CTAs of the LM-head kernel) x 4 lane quadrants
+    CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
     if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    const int G = ((cf.vocab + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N) * 4;
     argmax_merge_kernel<<<R, 256, 0, c->stream>>>(c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
@@ -515,7 +516,7 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
-    assemble_step_kernel<<<R, 128, 0, c->stream>>>(c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
+    assemble_step_kernel<<<R, 256, 0, c->stream>>>(c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
                                                    c->d_step_n, c->embed, cf.d_model, c->X);
   }
   int min_n = 1 << 30;
@@ -644,7 +645,7 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
     const int rows = last ? total - row0 : std::min(c->R_cap, total - last_rows - row0);
     {
       Launch l(c, TIDAR_TC_EMBED);
-      assemble_prefill_kernel<<<rows, 128, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
+      assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
                                                            cf.d_model, c->X);
     }
     if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64)) return rc;
