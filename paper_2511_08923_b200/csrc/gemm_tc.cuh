@@ -37,7 +37,10 @@ struct Args {
   int rb_rows;              // rows per row block: multiple of 16, 16..288
   int n_rb;                 // row blocks
   int n_tiles;              // ceil(N / 128)
-  int S;                    // K splits
+  int S;                    // K splits of the split region
+  int fused_items;          // items [0, fused_items) are whole tiles 0.. (no K split) finished by the mode's own epilogue;
+                            // the rest are tiles tile_b0.. split S ways along K, written as fp32 slabs
+  int tile_b0, n_tiles_b;   // first tile and tile count of the split region
   int kb_total;             // K / 64
   int stages;               // shared-memory ring depth
   int box_rows, n_box;      // activation rows per TMA box, boxes per stage
@@ -50,7 +53,23 @@ struct Args {
   // pre-fills the index table with -1); optional fp32 dump [R][ld_dump]
   float *cand_val; int32_t *cand_idx; float *dump; int ld_dump; int col0;
   int *status;              // device word set to 1 when a bounded wait gave up
+  __host__ __device__ int tile_b0_or_all() const { return n_tiles_b ? tile_b0 : n_tiles; }   // tiles per row block in the fused region
+  __host__ __device__ int total_items() const { return fused_items + n_rb * n_tiles_b * S; }
 };
+
+struct Item { int rb, tile, split, kb0, kb1; bool fused; };
+__device__ __forceinline__ Item decode_item(const Args &g, int item) {
+  Item w;
+  if (item < g.fused_items) {
+    w.fused = true; w.split = 0; w.tile = item % g.tile_b0_or_all(); w.rb = item / g.tile_b0_or_all();
+    w.kb0 = 0; w.kb1 = g.kb_total;
+  } else {
+    const int j = item - g.fused_items;
+    w.fused = false; w.split = j % g.S; w.tile = g.tile_b0 + (j / g.S) % g.n_tiles_b; w.rb = j / (g.S * g.n_tiles_b);
+    w.kb0 = (int)((long long)g.kb_total * w.split / g.S); w.kb1 = (int)((long long)g.kb_total * (w.split + 1) / g.S);
+  }
+  return w;
+}
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
 
@@ -66,7 +85,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
   const int a_stage_bytes = g.rb_rows * TILE_K * 2;
   const int stage_bytes = W_STAGE_BYTES + a_stage_bytes;            // multiple of 1024 (rb_rows % 16 == 0)
-  const int n_items = g.n_rb * g.n_tiles * g.S;
+  const int n_items = g.total_items();
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -94,9 +113,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint64_t pol_w = sm100::policy_evict_first(), pol_a = sm100::policy_evict_last();
       int s = 0; uint32_t ph = 0; bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const int split = item % g.S, tile = (item / g.S) % g.n_tiles, rb = item / (g.S * g.n_tiles);
-        const int kb0 = (int)((long long)g.kb_total * split / g.S), kb1 = (int)((long long)g.kb_total * (split + 1) / g.S);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        const Item w = decode_item(g, item);
+        const int tile = w.tile, rb = w.rb;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!sm100::mbar_wait(sm100::smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) { ok = false; break; }
           const uint32_t fb = sm100::smem_u32(&full_bar[s]);
           const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
@@ -123,8 +142,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       int s = 0; uint32_t ph = 0; bool ok = true; uint32_t it = 0;
       uint64_t wd = desc0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-        const int split = item % g.S;
-        const int kb0 = (int)((long long)g.kb_total * split / g.S), kb1 = (int)((long long)g.kb_total * (split + 1) / g.S);
+        const Item w = decode_item(g, item);
+        const int kb0 = w.kb0, kb1 = w.kb1;
         if (!sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp)) { ok = false; break; }
         sm100::tc_fence_after();
         uint32_t acc = 0u;
@@ -181,7 +200,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
     };
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-      const int split = item % g.S, tile = (item / g.S) % g.n_tiles, rb = item / (g.S * g.n_tiles);
+      const Item w = decode_item(g, item);
+      const int split = w.split, tile = w.tile, rb = w.rb;
       if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
       sm100::tc_fence_after();
       uint32_t v[9][16];
@@ -196,8 +216,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
       const int n = tile * TILE_N + q * 32 + lane;       // this thread's output feature
       const int r_base = rb * g.rb_rows + c_begin;
-      if (MODE == MODE_SLAB) {
-        float *o = g.out + (long long)split * g.slab_stride + n;
+      if (MODE == MODE_SLAB || !w.fused) {
+        // fp32 slab; columns are counted from the first tile of the split region
+        float *o = g.out + (long long)split * g.slab_stride + (n - g.tile_b0 * TILE_N);
         const bool n_ok = n < g.N;
 #pragma unroll
         for (int i = 0; i < 9; ++i) {

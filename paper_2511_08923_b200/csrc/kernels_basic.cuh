@@ -202,6 +202,21 @@ __global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16
   H[t] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
 }
 
+// SwiGLU over fp32 split-K slabs [S][R][ld] whose columns interleave (gate, up) and cover
+// features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).
+__global__ void swiglu_slab_kernel(const float *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
+                                   bf16 *__restrict__ H) {
+  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (size_t)R * nf) return;
+  const int r = (int)(t / nf), f = (int)(t % nf);
+  float g = 0.f, u = 0.f;
+  for (int s = 0; s < S; ++s) {
+    const float2 v = *reinterpret_cast<const float2 *>(slabs + s * stride + (size_t)r * ld + 2 * f);
+    g += v.x; u += v.y;
+  }
+  H[(size_t)r * ldh + f0 + f] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+}
+
 // Running per-row argmax over a chunk of logits [R][ncols] (fp32, leading dim ld)
 // that covers vocabulary ids [col0, col0+ncols).  Lowest index wins ties; NaN never
 // wins.  Optionally copies the chunk into a full [R][vocab] dump.

@@ -225,25 +225,49 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   gemm_tc::plan_rows(R, a);
   a.n_tiles = (N + gemm_tc::TILE_N - 1) / gemm_tc::TILE_N;
   a.kb_total = K / gemm_tc::TILE_K;
-  a.S = 1;
+  a.S = 1; a.fused_items = 0; a.tile_b0 = 0; a.n_tiles_b = 0;
+  int rem_tiles = 0;
   if (mode == gemm_tc::MODE_SLAB) {
+    a.n_tiles_b = a.n_tiles;
     a.S = force_S > 0 ? std::min(force_S, a.kb_total) : gemm_tc::plan_splits(a.n_rb * a.n_tiles, a.kb_total, c->n_sms, c->S_max, 4);
     a.out = slab_out ? slab_out : c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
   } else if (mode == gemm_tc::MODE_SWIGLU) {
     a.H = c->H; a.ldh = N / 2;
+    a.fused_items = a.n_rb * a.n_tiles;
+    // more tiles than SMs: whole waves of tiles finish in the fused epilogue; the tiles of the
+    // last, partial wave are split along K so that they also fill the machine, and are finished
+    // from fp32 slabs by swiglu_slab_kernel
+    if (a.n_rb == 1 && a.n_tiles > c->n_sms && a.n_tiles % c->n_sms) {
+      const int full = a.n_tiles / c->n_sms * c->n_sms;
+      const int rem = a.n_tiles - full;
+      const int S2 = std::min({c->n_sms / rem, a.kb_total / 4, c->S_max});
+      if (S2 >= 2 && (size_t)S2 * R * rem * gemm_tc::TILE_N <= c->partials_cap) {
+        rem_tiles = rem;
+        a.fused_items = full; a.tile_b0 = full; a.n_tiles_b = rem; a.S = S2;
+        a.out = c->partials; a.ldo = rem * gemm_tc::TILE_N; a.slab_stride = (long long)R * a.ldo;
+      }
+    }
   } else {
+    a.fused_items = a.n_rb * a.n_tiles;
     a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.dump = c->dbg_logits; a.ld_dump = c->cfg.vocab; a.col0 = 0;
   }
   a.status = c->d_status;
   const CUtensorMap *tmA = act_map(c, A, a_rows, K, a.box_rows);
   if (!tmA) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for an activation matrix (%d x %d, box %d)", a_rows, K, a.box_rows);
-  const int items = a.n_rb * a.n_tiles * a.S;
+  const int items = a.total_items();
   const int grid = std::min(items, c->n_sms);
   const size_t smem = gemm_tc::smem_bytes(a);
   Launch l(c, cls);
   if (mode == gemm_tc::MODE_SLAB) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
   else if (mode == gemm_tc::MODE_SWIGLU) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
   else gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  if (rem_tiles) {
+    const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
+    const size_t n = (size_t)R * nf;
+    c->launches++;
+    swiglu_slab_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
+  }
   if (S_out) *S_out = a.S;
   if (stride_out) *stride_out = (size_t)R * N;
   return TIDAR_OK;

@@ -242,3 +242,30 @@ def test_errors_are_reported_before_launch(impl):
     with pytest.raises(TidarError):
         t.step([0], forced=[9])
     t.close()
+
+
+@pytest.mark.parametrize("name,over", [
+    # 2*d_ffn/128 = 151 weight tiles > 148 SMs: whole-wave tiles fused, leftover tiles K-split
+    ("wide_ffn", dict(d_model=1024, n_q_heads=8, n_kv_heads=2, head_dim=128, d_ffn=9664, n_layers=1, vocab=1024)),
+    # six query heads per KV head (the 1.5B-class grouping): 21 slots x 6 heads per attention tile
+    ("group6", dict(d_model=768, n_q_heads=6, n_kv_heads=1, head_dim=128, d_ffn=1024, n_layers=2, vocab=2048)),
+])
+def test_other_shapes_prefill_and_steps(name, over):
+    from dataclasses import replace
+    from tidar_synth import CONFIGS, gen_model_weights
+    sh = replace(CONFIGS["tiny"], name=name, tie_lm_head=False, k=8, **over)
+    wt = gen_model_weights(sh)
+    cfg, w = oracle_cfg(sh), O.weights_to_f64(wt)
+    prompt = prompt_ids(sh, 70)
+    k = sh.k
+    t = _gpu(sh, wt, 0, max_seq_len=256)
+    t.prefill(0, prompt, k)
+    st, c, fo = O.prefill(cfg, w, prompt, k, return_forward=True)
+    _compare_pass(t, fo, np.arange(len(prompt) + k))
+    for s in range(2):
+        t.set_block(0, st.block)
+        so = O.step(cfg, w, st, forced=3)
+        toks, Ls = t.step([0], forced=[3])
+        _compare_pass(t, so.fwd, np.arange(k * (k + 1)))
+        assert Ls == [3]
+    t.close()
