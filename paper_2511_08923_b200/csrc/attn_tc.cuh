@@ -74,6 +74,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag, sh_max_nvis, sh_loc_lo, sh_loc_hi;
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
 
@@ -106,6 +107,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     sm100::tmem_relinquish();
   }
   __syncthreads();
+  pdl_wait();                 // everything below reads what earlier kernels of the pass wrote
 
   // ---- per-row metadata (softmax threads own one MMA row each) and the tile's key range ----
   const int my_row = (warp & 3) * 32 + lane;             // MMA row = TMEM lane (softmax warps only)
@@ -370,6 +372,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
                                bf16 *__restrict__ O) {
+  pdl_trigger();
+  pdl_wait();
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (wid >= R * Hq) return;
   float M = -INFINITY;

@@ -44,3 +44,12 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
+
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization
+// attribute may start while the previous kernel of the stream is still running;
+// pdl_wait() blocks until that kernel has completed and its writes are visible, so
+// everything before it may only touch data no earlier kernel writes (weights, the
+// kernel's own shared / tensor memory).  pdl_trigger() lets the next kernel of the stream
+// be scheduled early in the same way.  Both are no-ops in a plain launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

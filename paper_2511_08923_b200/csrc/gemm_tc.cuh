@@ -81,6 +81,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
   const int a_stage_bytes = g.rb_rows * TILE_K * 2;
@@ -112,15 +113,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       sm100::prefetch_tensormap(&tmA);
       const uint64_t pol_w = sm100::policy_evict_first(), pol_a = sm100::policy_evict_last();
       int s = 0; uint32_t ph = 0; bool ok = true;
+      // Weights are never written by a kernel, so the first stages' weight tiles are requested
+      // before waiting for the previous kernel; their activation tiles follow the wait.
+      int pre = 0;
+      if ((int)blockIdx.x < n_items) {
+        const Item w0 = decode_item(g, blockIdx.x);
+        pre = min(g.stages, w0.kb1 - w0.kb0);
+        for (int i = 0; i < pre; ++i) {
+          const uint32_t fb = sm100::smem_u32(&full_bar[i]);
+          sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
+          sm100::tma_load_2d(smem0 + (uint32_t)i * stage_bytes, &tmW, fb, (w0.kb0 + i) * TILE_K, w0.tile * TILE_N, pol_w);
+        }
+      }
+      pdl_wait();
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item w = decode_item(g, item);
         const int tile = w.tile, rb = w.rb;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
-          if (!sm100::mbar_wait(sm100::smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) { ok = false; break; }
           const uint32_t fb = sm100::smem_u32(&full_bar[s]);
           const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
-          sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
-          sm100::tma_load_2d(sw, &tmW, fb, kb * TILE_K, tile * TILE_N, pol_w);
+          if (pre > 0) {
+            --pre;                                   // weights of this stage are already on their way
+          } else {
+            if (!sm100::mbar_wait(sm100::smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) { ok = false; break; }
+            sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
+            sm100::tma_load_2d(sw, &tmW, fb, kb * TILE_K, tile * TILE_N, pol_w);
+          }
           for (int b = 0; b < g.n_box; ++b)
             sm100::tma_load_2d(sa + (uint32_t)(b * g.box_rows * TILE_K * 2), &tmA, fb, kb * TILE_K, rb * g.rb_rows + b * g.box_rows, pol_a);
           if (++s == g.stages) { s = 0; ph ^= 1u; }
@@ -175,6 +193,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else {
     // ===================== epilogue =====================
+    pdl_wait();
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;
     const int hc = ((g.rb_rows / 2 + 15) / 16) * 16;

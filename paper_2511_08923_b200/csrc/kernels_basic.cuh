@@ -27,6 +27,8 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
                                      const int32_t *__restrict__ block_ids, int k, int k_max, int mask_id,
                                      int32_t *__restrict__ step_n, const bf16 *__restrict__ embed, int d,
                                      float *__restrict__ X) {
+  pdl_trigger();
+  pdl_wait();
   const int T = k * (k + 1);
   const int r = blockIdx.x;
   const int s = r / T, slot = r % T;
@@ -90,6 +92,8 @@ __global__ void attn_meta_kernel(RowMeta m, const int32_t *__restrict__ seq_len,
 // layer and head), stored as float.
 __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int R, int half, double theta,
                                   float *__restrict__ cs, float *__restrict__ sn) {
+  pdl_trigger();
+  pdl_wait();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= R * half) return;
   const int r = t / half, i = t % half;
@@ -108,6 +112,8 @@ template <int THREADS>
 __global__ void __launch_bounds__(THREADS)
 rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials, int S, size_t partial_stride,
                       const bf16 *__restrict__ gain, float eps, int d, bf16 *__restrict__ A) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float row[];
   __shared__ float red[THREADS / 32];
   const int r = blockIdx.x;
@@ -152,6 +158,8 @@ rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride,
                RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
                bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
                bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
+  pdl_trigger();
+  pdl_wait();
   // one block per row; a work unit is 4 consecutive dims i..i+3 of the first half of one
   // head together with their rotation partners i+hd/2..
   const int r = blockIdx.x, half = hd / 2, upr = half / 4;          // units per head
@@ -206,6 +214,8 @@ __global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16
 // features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).
 __global__ void swiglu_slab_kernel(const float *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
                                    bf16 *__restrict__ H) {
+  pdl_trigger();
+  pdl_wait();
   const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= (size_t)R * nf) return;
   const int r = (int)(t / nf), f = (int)(t % nf);
@@ -256,6 +266,8 @@ __global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int nco
 // order in which candidates are combined.
 __global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t *__restrict__ pi, int G, int R,
                                     float *__restrict__ best_val, int32_t *__restrict__ best_idx) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   float bv = -INFINITY; int bi = 0x7fffffff;
   for (int g = threadIdx.x; g < G; g += blockDim.x) {
@@ -300,6 +312,8 @@ __global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const 
                                      const int32_t *__restrict__ forced, int k, int k_max,
                                      int32_t *__restrict__ block_ids, int32_t *__restrict__ step_L,
                                      int32_t *__restrict__ out /*[n_seqs][k_max+1]*/) {
+  pdl_trigger();
+  pdl_wait();
   const int s = blockIdx.x, lane = threadIdx.x;
   const int T = k * (k + 1);
   const int seq = step_seqs[s];
@@ -348,6 +362,8 @@ __global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int r
 __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ step_n,
                                  const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, int poison,
                                  KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride) {
+  pdl_trigger();
+  pdl_wait();
   const int s = blockIdx.x, l = blockIdx.y;
   const int seq = step_seqs[s];
   const int n = step_n[s], L = step_L[s];

@@ -177,6 +177,20 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   *bytes = align_up(cv.off, 256);
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the
+// previous kernel of the stream is still running and synchronises itself with pdl_wait().
+// Only kernels that call pdl_wait() before touching produced data may be launched this way.
+template <typename... KP, typename... AP>
+inline void launch_pdl(void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AP &&...args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, KP(std::forward<AP>(args))...);
+}
+
 // ---- launch bookkeeping -----------------------------------------------------
 struct Launch {
   tidar_ctx *c; int cls; cudaEvent_t a = nullptr, b = nullptr;
@@ -258,14 +272,14 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   const int grid = std::min(items, c->n_sms);
   const size_t smem = gemm_tc::smem_bytes(a);
   Launch l(c, cls);
-  if (mode == gemm_tc::MODE_SLAB) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
-  else if (mode == gemm_tc::MODE_SWIGLU) gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
-  else gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX><<<grid, gemm_tc::THREADS, smem, c->stream>>>(tmW, *tmA, a);
+  if (mode == gemm_tc::MODE_SLAB) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
+  else if (mode == gemm_tc::MODE_SWIGLU) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
+  else launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
   if (rem_tiles) {
     const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
     const size_t n = (size_t)R * nf;
     c->launches++;
-    swiglu_slab_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+    launch_pdl(swiglu_slab_kernel, (unsigned)((n + 255) / 256), 256, 0, c->stream, c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
                                                                            a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
   }
   if (S_out) *S_out = a.S;
@@ -338,17 +352,17 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   {
     Launch l(c, TIDAR_TC_ATTN);
     if (cf.head_dim == 128)
-      attn_tc::attn_tc_kernel<128><<<grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      launch_pdl(attn_tc::attn_tc_kernel<128>, grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
     else
-      attn_tc::attn_tc_kernel<64><<<grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream>>>(*m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      launch_pdl(attn_tc::attn_tc_kernel<64>, grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
   }
   if (a.splits > 1) {
     Launch l(c, TIDAR_TC_ATTN);
     const int warps = R * cf.n_q_heads;
     if (cf.head_dim == 128)
-      attn_tc::attn_combine_kernel<128><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_pdl(attn_tc::attn_combine_kernel<128>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
     else
-      attn_tc::attn_combine_kernel<64><<<(warps + 7) / 8, 256, 0, c->stream>>>(c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_pdl(attn_tc::attn_combine_kernel<64>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
   }
 }
 
@@ -366,7 +380,7 @@ void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *V
 void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t stride, const bf16 *gain) {
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
-  rmsnorm_reduce_kernel<512><<<R, 512, d * sizeof(float), c->stream>>>(c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+  launch_pdl(rmsnorm_reduce_kernel<512>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
 }
 
 // The transformer stack over R assembled rows (metadata and X already filled).
@@ -378,7 +392,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
   {
     Launch l(c, TIDAR_TC_ROPE);
     const int n = R * (hd / 2);
-    rope_table_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
+    launch_pdl(rope_table_kernel, (n + 255) / 256, 256, 0, c->stream, c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
   }
   int S = 0; size_t stride = 0;          // pending partials of the previous down projection
   const bool tc = cf.impl == 0;
@@ -393,7 +407,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
-      rope_kv_kernel<<<R, 256, 0, c->stream>>>(c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+      launch_pdl(rope_kv_kernel, R, 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     if (tc) {
@@ -423,7 +437,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
     if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    argmax_merge_kernel<<<R, 256, 0, c->stream>>>(c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
+    launch_pdl(argmax_merge_kernel, R, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
@@ -540,7 +554,7 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
-    assemble_step_kernel<<<R, 256, 0, c->stream>>>(c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
+    launch_pdl(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
                                                    c->d_step_n, c->embed, cf.d_model, c->X);
   }
   int min_n = 1 << 30;
@@ -549,12 +563,12 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   if (rc) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    verify_select_kernel<<<n_seqs, 32, 0, c->stream>>>(c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
+    launch_pdl(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
                                                        c->d_step_L, c->d_out);
   }
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    kv_commit_kernel<<<dim3(n_seqs, cf.n_layers), 128, 0, c->stream>>>(c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
+    launch_pdl(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
                                                                        (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
   }
   CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
