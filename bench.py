@@ -78,7 +78,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                       "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.p = None
         return self
@@ -220,7 +220,7 @@ def workload_config(sh, k, n0, batch):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=list(CONFIGS))
@@ -342,7 +342,12 @@ def main():
         t_tensor = cost["flops"] / (pk["bf16_tflops_sustained"] * 1e12) * 1e3
         t_hbm_nom = cost["bytes"] / (NOMINAL["hbm_gbs"] * 1e9) * 1e3
         t_tensor_nom = cost["flops"] / (NOMINAL["bf16_tflops"] * 1e12) * 1e3
+        # Dominant kernel: gemm_tc_kernel (every projection and the LM head; three epilogue
+        # variants of one kernel).  Its launches of one step are timed one by one with CUDA
+        # events on the library's stream (classes "gemm" and "lmhead"; the LM-head class also
+        # holds the small argmax merge kernel).
         gemm_ms = cls.get("gemm", 0.0) + cls.get("lmhead", 0.0)
+        n_gemm_launches = 4 * sh.n_layers + 1
         tensor_bound = t_tensor >= t_hbm
         if tensor_bound:
             ach = cost["gemm_flops"] / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
@@ -350,9 +355,13 @@ def main():
         else:
             ach = cost["weight_bytes"] / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
             roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s"}
-        roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": TRAFFIC_NOTE.get(args.workload),
-                     "kernel": "projection GEMMs (QKV, O, gate/up, down, LM head) summed over one step",
-                     "peak_source": pk_src + (" (sustained bf16)" if tensor_bound else " (copy bandwidth)"),
+        tr = TRAFFIC.get(args.workload)
+        roof.update({"frac": roof["achieved"] / roof["peak"],
+                     "traffic": tr["bytes_per_step"] if tr else None,
+                     "traffic_note": tr["note"] if tr else "no ncu capture of this workload since the kernel last changed",
+                     "kernel": f"gemm_tc_kernel, all {n_gemm_launches} launches of one step (QKV, O, gate/up, down per layer + LM head)",
+                     "algorithmic": {"flops_per_step": cost["gemm_flops"], "weight_bytes_per_step": cost["weight_bytes"]},
+                     "peak_source": pk_src + (" (bf16 matmul, sustained: the kernel runs inside a long step)" if tensor_bound else " (copy bandwidth)"),
                      "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {a: round(b, 4) for a, b in cls.items()}})
         line = {"metric": "decode_tokens_per_s", "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -383,8 +392,10 @@ def main():
 
 
 DEFAULT_IMPL = 0
-# dram bytes per step of the projection kernels from an ncu capture (see profiles/); None until captured
-TRAFFIC_NOTE = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of gemm_tc_kernel per step, from the ncu capture
+# summarised in profiles/ (2-layer twin of the workload; per-layer traffic x n_layers + the LM
+# head launch).  Removed whenever the kernel changes after the capture.
+TRAFFIC = {}
 
 if __name__ == "__main__":
     main()
