@@ -11,13 +11,15 @@
 //
 // Tiling: the G = Hq/Hkv query heads that share a KV head are packed into one 128-row
 // MMA tile (floor(128/G) slots x G heads), so K/V are read once per KV head.  Per key
-// tile: S = Q K^T (M 128, N 64, K hd) into TMEM; the softmax warps read S (one thread per
-// row), keep the running max / sum, write P (bf16) to shared memory in the MMA operand
-// layout; O_tile = P V (M 128, N hd, K 64, V as the MN-major operand) into TMEM; the
-// softmax warps add it to their register accumulator.  S, P and O_tile are double
-// buffered, so QK^T of tile t+1 runs while tile t is in softmax.  The key range of a query
-// tile can be split over several CTAs; partial (max, sum, O) results are merged by
-// attn_combine_kernel.
+// tile: S = Q K^T (M 128, N 64, K hd) into TMEM (double buffered); the softmax warps read S
+// (one thread per row), keep a reference max and the running sum, write P (bf16) to shared
+// memory in the MMA operand layout; O += P V (M 128, N hd, K 64, V as the MN-major operand)
+// accumulates in TMEM over all key tiles.  The reference max is only raised when a tile
+// exceeds it by more than 2^8 (P stays <= 256, exact enough in bf16/fp32); raising it
+// rescales the rows of O in TMEM, which happens in the first tiles only.  The CTA needs
+// <= 113 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
+// share an SM and fill each other's dependency stalls.  The key range of a query tile can be
+// split over several CTAs; partial (max, sum, O) results are merged by attn_combine_kernel.
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -25,9 +27,10 @@
 namespace attn_tc {
 
 constexpr int KT = 64;               // keys per tile (= page size)
-constexpr int KV_STAGES = 3;
+constexpr int KV_STAGES = 2;
 constexpr int THREADS = 192;         // warp 0: TMA, warp 1: MMA, warps 2..5: softmax
 constexpr int MAX_SPLITS = 8;
+constexpr float RAISE_THRESHOLD = 8.f;   // log2 units
 
 struct Args {
   int R;                    // rows (slots) of the pass
@@ -44,10 +47,11 @@ struct Args {
   bf16 *O;                                   // [R][Hq*hd]
   float *part_O;                             // [splits][R][Hq][hd]  (splits > 1)
   float *part_ml;                            // [splits][R][Hq][2]
-  unsigned long long *tile_stats;            // [2]: key tiles issued, key tiles a dense-mask kernel would issue (may be null)
   int *status;
 };
 
+// Shared memory of one CTA; everything is dynamic so that the 1024-byte alignment the
+// swizzled tiles need costs no padding (the kernel checks the base address).
 template <int HD>
 struct Smem {
   static constexpr int NH = HD / 64;                 // 64-element halves of a head
@@ -58,25 +62,33 @@ struct Smem {
   static constexpr int K_OFF = Q_OFF + Q_BYTES;
   static constexpr int V_OFF = K_OFF + KV_STAGES * KV_BYTES;
   static constexpr int P_OFF = V_OFF + KV_STAGES * KV_BYTES;
-  static constexpr int TOTAL = P_OFF + 2 * P_BYTES + 1024;
-  static constexpr int TMEM_COLS = HD == 128 ? 512 : 256;      // 2 x 64 (S) + 2 x HD (O), rounded up to a power of two
+  static constexpr int BAR_OFF = P_OFF + P_BYTES;    // mbarriers and a few words
+  static constexpr int TOTAL = BAR_OFF + 256;
+  static constexpr int TMEM_COLS = 256;              // 2 x 64 (S) + HD (O) <= 256
 };
 
+struct Ctl {                                         // lives at Smem::BAR_OFF
+  uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES], s_full[2], s_empty[2], p_full, p_empty;
+  uint32_t tmem_base;
+  int abort_flag, max_nvis, loc_lo, loc_hi;
+};
+static_assert(sizeof(Ctl) <= 256, "control block must fit its slot");
+
 template <int HD>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-       const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a) {
+               const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a) {
   using L = Smem<HD>;
   constexpr int NH = L::NH;
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES],
-      s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2];
-  __shared__ uint32_t tmem_base_slot;
-  __shared__ int abort_flag, sh_max_nvis, sh_loc_lo, sh_loc_hi;
-
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t smem0 = sm100::smem_u32(smem_raw);
+  if (smem0 & 1023u) {                               // cannot place swizzled tiles: report, touch nothing
+    if (threadIdx.x == 0 && a.status) atomicExch(a.status, 3);
+    return;
+  }
+  Ctl &ctl = *reinterpret_cast<Ctl *>(smem_raw + L::BAR_OFF);
 
   // ---- which work item ----
   int w = blockIdx.x;
@@ -88,22 +100,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   const int rows_used = a.spt * a.G;                                   // MMA rows that carry data
 
   if (threadIdx.x == 0) {
-    abort_flag = 0; sh_max_nvis = 0; sh_loc_lo = 0x7fffffff; sh_loc_hi = 0;
-    sm100::mbar_init(sm100::smem_u32(&q_full), 1);
+    ctl.abort_flag = 0; ctl.max_nvis = 0; ctl.loc_lo = 0x7fffffff; ctl.loc_hi = 0;
+    sm100::mbar_init(sm100::smem_u32(&ctl.q_full), 1);
     for (int s = 0; s < KV_STAGES; ++s) {
-      sm100::mbar_init(sm100::smem_u32(&k_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&k_empty[s]), 1);
-      sm100::mbar_init(sm100::smem_u32(&v_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&v_empty[s]), 1);
+      sm100::mbar_init(sm100::smem_u32(&ctl.k_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.k_empty[s]), 1);
+      sm100::mbar_init(sm100::smem_u32(&ctl.v_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.v_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      sm100::mbar_init(sm100::smem_u32(&s_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&s_empty[b]), 4);
-      sm100::mbar_init(sm100::smem_u32(&p_full[b]), 4); sm100::mbar_init(sm100::smem_u32(&p_empty[b]), 1);
-      sm100::mbar_init(sm100::smem_u32(&o_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&o_empty[b]), 4);
-    }
+    for (int b = 0; b < 2; ++b) { sm100::mbar_init(sm100::smem_u32(&ctl.s_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.s_empty[b]), 4); }
+    sm100::mbar_init(sm100::smem_u32(&ctl.p_full), 4); sm100::mbar_init(sm100::smem_u32(&ctl.p_empty), 1);
     sm100::fence_mbar_init();
   }
   if (warp == 1) {
     __syncwarp();
-    sm100::tmem_alloc(sm100::smem_u32(&tmem_base_slot), L::TMEM_COLS);
+    sm100::tmem_alloc(sm100::smem_u32(&ctl.tmem_base), L::TMEM_COLS);
     sm100::tmem_relinquish();
   }
   __syncthreads();
@@ -118,55 +127,53 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (sl < a.spt && pr < row_end) {
       my_slot = pr; my_head = kvh * a.G + my_row % a.G;
       my_nvis = a.nvis[pr]; my_nloc = a.nloc[pr]; my_loc0 = a.loc0[pr];
-      atomicMax(&sh_max_nvis, my_nvis);
-      if (my_nloc > 0) { atomicMin(&sh_loc_lo, my_loc0); atomicMax(&sh_loc_hi, my_loc0 + my_nloc); }
+      atomicMax(&ctl.max_nvis, my_nvis);
+      if (my_nloc > 0) { atomicMin(&ctl.loc_lo, my_loc0); atomicMax(&ctl.loc_hi, my_loc0 + my_nloc); }
     }
   }
   sm100::tc_fence_before();
   __syncthreads();
   sm100::tc_fence_after();
-  const uint32_t tmem = tmem_base_slot;
-  const uint32_t tmem_S = tmem, tmem_O = tmem + 2 * KT;               // S: 2 x 64 columns, O: 2 x HD columns
-  const int max_nvis = sh_max_nvis;
-  const int loc_lo = sh_loc_lo, loc_hi = sh_loc_hi;
+  const uint32_t tmem = ctl.tmem_base;
+  const uint32_t tmem_S = tmem, tmem_O = tmem + 2 * KT;               // S: 2 x 64 columns, O: HD columns
+  const int max_nvis = ctl.max_nvis;
+  const int loc_lo = ctl.loc_lo, loc_hi = ctl.loc_hi;
   const int n_cache_tiles = (max_nvis + KT - 1) / KT;
   const int n_loc_tiles = loc_hi > loc_lo ? (loc_hi - loc_lo + KT - 1) / KT : 0;
   const int nt_all = n_cache_tiles + n_loc_tiles;
   const int t_begin = (int)((long long)nt_all * sp / a.splits), t_end = (int)((long long)nt_all * (sp + 1) / a.splits);
   const int nt = t_end - t_begin;
   const int seq = row0 < a.R ? a.seq[row0] : 0;
-  volatile int *abortp = &abort_flag;
+  volatile int *abortp = &ctl.abort_flag;
 
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0 && nt > 0) {
-      const uint64_t pol_q = sm100::policy_evict_last(), pol_kv = sm100::policy_evict_last();
-      const uint32_t qb = sm100::smem_u32(&q_full);
+      const uint64_t pol = sm100::policy_evict_last();
+      const uint32_t qb = sm100::smem_u32(&ctl.q_full);
       sm100::mbar_expect_tx(qb, (uint32_t)(NH * rows_used * 128));
       for (int h = 0; h < NH; ++h)
-        sm100::tma_load_3d(smem0 + L::Q_OFF + h * (128 * 128), &tmQ, qb, h * 64, kvh * a.G, row0, pol_q);
+        sm100::tma_load_3d(smem0 + L::Q_OFF + h * (128 * 128), &tmQ, qb, h * 64, kvh * a.G, row0, pol);
       int s = 0; uint32_t ph = 0; bool ok = true;
       for (int t = t_begin; t < t_end && ok; ++t) {
         const bool is_cache = t < n_cache_tiles;
         const int page = is_cache ? a.page_table[(size_t)seq * a.pages_per_seq + t] : 0;
         const int lrow = loc_lo + (t - n_cache_tiles) * KT;
-        // K
-        if (!sm100::mbar_wait(sm100::smem_u32(&k_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
-        uint32_t fb = sm100::smem_u32(&k_full[s]);
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.k_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+        uint32_t fb = sm100::smem_u32(&ctl.k_full[s]);
         sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
         for (int h = 0; h < NH; ++h) {
           const uint32_t dst = smem0 + L::K_OFF + s * L::KV_BYTES + h * (KT * 128);
-          if (is_cache) sm100::tma_load_4d(dst, &tmK, fb, h * 64, 0, kvh, a.page_base_k + page, pol_kv);
-          else sm100::tma_load_3d(dst, &tmKloc, fb, h * 64, kvh, lrow, pol_kv);
+          if (is_cache) sm100::tma_load_4d(dst, &tmK, fb, h * 64, 0, kvh, a.page_base_k + page, pol);
+          else sm100::tma_load_3d(dst, &tmKloc, fb, h * 64, kvh, lrow, pol);
         }
-        // V
-        if (!sm100::mbar_wait(sm100::smem_u32(&v_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
-        fb = sm100::smem_u32(&v_full[s]);
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.v_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+        fb = sm100::smem_u32(&ctl.v_full[s]);
         sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
         for (int h = 0; h < NH; ++h) {
           const uint32_t dst = smem0 + L::V_OFF + s * L::KV_BYTES + h * (KT * 128);
-          if (is_cache) sm100::tma_load_4d(dst, &tmV, fb, h * 64, 0, kvh, a.page_base_v + page, pol_kv);
-          else sm100::tma_load_3d(dst, &tmVloc, fb, h * 64, kvh, lrow, pol_kv);
+          if (is_cache) sm100::tma_load_4d(dst, &tmV, fb, h * 64, 0, kvh, a.page_base_v + page, pol);
+          else sm100::tma_load_3d(dst, &tmVloc, fb, h * 64, kvh, lrow, pol);
         }
         if (++s == KV_STAGES) { s = 0; ph ^= 1u; }
       }
@@ -176,20 +183,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (lane == 0 && nt > 0) {
       const uint32_t idesc_qk = sm100::make_idesc_bf16(128, KT);
       const uint32_t idesc_pv = sm100::make_idesc_bf16(128, HD) | (1u << 16);      // B (= V) is MN-major
-      bool ok = sm100::mbar_wait(sm100::smem_u32(&q_full), 0, abortp);
+      bool ok = sm100::mbar_wait(sm100::smem_u32(&ctl.q_full), 0, abortp);
       sm100::tc_fence_after();
       int ks = 0; uint32_t kph = 0;          // K ring position of the next QK^T
       int vs = 0; uint32_t vph = 0;          // V ring position of the next PV
       // descriptors are built once; the issue loop only adds 16-byte-unit offsets
       const uint64_t q_desc = sm100::make_desc_sw128(smem0 + L::Q_OFF);
       const uint64_t k_desc0 = sm100::make_desc_sw128(smem0 + L::K_OFF);
-      const uint64_t p_desc0 = sm100::make_desc_sw128(smem0 + L::P_OFF);
+      const uint64_t p_desc = sm100::make_desc_sw128(smem0 + L::P_OFF);
       const uint64_t v_desc0 = sm100::make_desc_sw128_mn(smem0 + L::V_OFF, KT * 128);
-      constexpr uint64_t KV16 = L::KV_BYTES >> 4, P16 = L::P_BYTES >> 4;
+      constexpr uint64_t KV16 = L::KV_BYTES >> 4;
       auto issue_qk = [&](int i) -> bool {   // i: tile counter of this CTA
         const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
-        if (!sm100::mbar_wait(sm100::smem_u32(&k_full[ks]), kph, abortp)) return false;
-        if (!sm100::mbar_wait(sm100::smem_u32(&s_empty[b]), bph ^ 1u, abortp)) return false;
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.k_full[ks]), kph, abortp)) return false;
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.s_empty[b]), bph ^ 1u, abortp)) return false;
         sm100::tc_fence_after();
         const uint64_t kd = k_desc0 + (uint64_t)ks * KV16;
         const uint32_t d = tmem_S + b * KT;
@@ -199,64 +206,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           sm100::mma_bf16_ss(d, q_desc + (kk / 4) * (128 * 128 / 16) + (kk % 4) * 2, kd + (kk / 4) * (KT * 128 / 16) + (kk % 4) * 2, idesc_qk,
                              kk > 0 ? 1u : 0u);
         }
-        sm100::mma_commit(sm100::smem_u32(&k_empty[ks]));
-        sm100::mma_commit(sm100::smem_u32(&s_full[b]));
+        sm100::mma_commit(sm100::smem_u32(&ctl.k_empty[ks]));
+        sm100::mma_commit(sm100::smem_u32(&ctl.s_full[b]));
         if (++ks == KV_STAGES) { ks = 0; kph ^= 1u; }
         return true;
       };
       if (ok) ok = issue_qk(0);
       for (int i = 0; i < nt && ok; ++i) {
         if (i + 1 < nt) { ok = issue_qk(i + 1); if (!ok) break; }
-        const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
-        if (!sm100::mbar_wait(sm100::smem_u32(&v_full[vs]), vph, abortp)) { ok = false; break; }
-        if (!sm100::mbar_wait(sm100::smem_u32(&o_empty[b]), bph ^ 1u, abortp)) { ok = false; break; }
-        if (!sm100::mbar_wait(sm100::smem_u32(&p_full[b]), bph, abortp)) { ok = false; break; }
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.v_full[vs]), vph, abortp)) { ok = false; break; }
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.p_full), (uint32_t)i & 1u, abortp)) { ok = false; break; }
         sm100::tc_fence_after();
-        const uint64_t pd = p_desc0 + (uint64_t)b * P16;
         const uint64_t vd = v_desc0 + (uint64_t)vs * KV16;
-        const uint32_t d = tmem_O + b * HD;
 #pragma unroll
         for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per instruction: 32 B along a P row, 16 V rows (2048 B)
-          sm100::mma_bf16_ss(d, pd + kk * 2, vd + kk * (16 * 128 / 16), idesc_pv, kk > 0 ? 1u : 0u);
-        sm100::mma_commit(sm100::smem_u32(&v_empty[vs]));
-        sm100::mma_commit(sm100::smem_u32(&p_empty[b]));
-        sm100::mma_commit(sm100::smem_u32(&o_full[b]));
+          sm100::mma_bf16_ss(tmem_O, p_desc + kk * 2, vd + kk * (16 * 128 / 16), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+        sm100::mma_commit(sm100::smem_u32(&ctl.v_empty[vs]));
+        sm100::mma_commit(sm100::smem_u32(&ctl.p_empty));      // P consumed and O up to date through tile i
         if (++vs == KV_STAGES) { vs = 0; vph ^= 1u; }
       }
     }
   } else {
-    // ===================== softmax + accumulation =====================
+    // ===================== softmax =====================
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    float o_acc[HD];
-#pragma unroll
-    for (int d = 0; d < HD; ++d) o_acc[d] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f, m_acc = -INFINITY, m_prev = -INFINITY;
+    float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
-
-    auto accumulate = [&](int i, float m_tile) -> bool {       // add O_tile(i), computed under max m_tile
-      const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
-      if (!sm100::mbar_wait(sm100::smem_u32(&o_full[b]), bph, abortp)) return false;
-      sm100::tc_fence_after();
-      const float f = (m_acc == -INFINITY) ? 0.f : exp2f(m_acc - m_tile);
-#pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t v[32];
-        sm100::tmem_ld32(tmem_O + lane_addr + b * HD + c * 32, v);
-        sm100::tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o_acc[c * 32 + j] = fmaf(o_acc[c * 32 + j], f, __uint_as_float(v[j]));
-      }
-      sm100::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&o_empty[b]));
-      m_acc = m_tile;
-      return true;
-    };
-
     for (int i = 0; i < nt && ok; ++i) {
       const int t = t_begin + i;
       const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
-      if (!sm100::mbar_wait(sm100::smem_u32(&s_full[b]), bph, abortp)) { ok = false; break; }
+      if (!sm100::mbar_wait(sm100::smem_u32(&ctl.s_full[b]), bph, abortp)) { ok = false; break; }
       sm100::tc_fence_after();
       uint32_t sv[64];
       {
@@ -269,7 +247,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       }
       sm100::tc_fence_before();
       __syncwarp();
-      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&s_empty[b]));
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&ctl.s_empty[b]));
 
       // visible keys of this tile for my row: [lo, hi) in tile-local indices
       int lo = 0, hi = 0;
@@ -288,9 +266,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         sv[j] = __float_as_uint(s);
         mx = fmaxf(mx, s);
       }
-      const float m_new = fmaxf(m_run, mx);
+      // raise the reference only when this tile exceeds it by more than the threshold
+      // (-inf + threshold = -inf, so the first visible key always sets it)
+      const float m_new = (mx > m_ref + RAISE_THRESHOLD) ? mx : m_ref;
+      const float alpha = (m_new == m_ref) ? 1.f : exp2f(m_ref - m_new);      // m_ref = -inf gives 0
       const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-      const float alpha = exp2f(m_run - m_safe);              // m_run = -inf gives 0
       float sum = 0.f;
       uint32_t pk[32];
 #pragma unroll
@@ -301,12 +281,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         pk[j >> 1] = *reinterpret_cast<uint32_t *>(&h2);
       }
       l_run = l_run * alpha + sum;
-      m_run = m_new;
+      m_ref = m_new;
 
+      // PV of the previous tile must be complete: it read P and updated O
+      if (!sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), ((uint32_t)i & 1u) ^ 1u, abortp)) { ok = false; break; }
+      if (i > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        sm100::tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t v[32];
+          sm100::tmem_ld32(tmem_O + lane_addr + c * 32, v);
+          sm100::tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+          sm100::tmem_st32(tmem_O + lane_addr + c * 32, v);
+        }
+        sm100::tmem_wait_st();
+        sm100::tc_fence_before();
+      }
       // P -> shared memory in the 128-byte-swizzled K-major operand layout
-      if (!sm100::mbar_wait(sm100::smem_u32(&p_empty[b]), bph ^ 1u, abortp)) { ok = false; break; }
       {
-        const uint32_t prow = smem0 + L::P_OFF + b * L::P_BYTES + (my_row >> 3) * 1024 + (my_row & 7) * 128;
+        const uint32_t prow = smem0 + L::P_OFF + (my_row >> 3) * 1024 + (my_row & 7) * 128;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           const uint32_t dst = prow + ((c ^ (my_row & 7)) << 4);
@@ -316,46 +311,52 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       }
       sm100::fence_proxy_async();
       __syncwarp();
-      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&p_full[b]));
-
-      if (i >= 1) ok = accumulate(i - 1, m_prev);
-      m_prev = m_run;
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&ctl.p_full));
     }
-    if (ok && nt > 0) ok = accumulate(nt - 1, m_prev);
-
-    // ---- output ----
-    if (ok && my_slot >= 0) {
-      if (a.splits == 1) {
-        const float inv = 1.f / l_run;
-        bf16 *o = a.O + ((size_t)my_slot * a.Hq + my_head) * HD;
+    // ---- output: O is complete once the last PV has finished ----
+    if (ok && nt > 0) ok = sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), (uint32_t)(nt - 1) & 1u, abortp);
+    if (ok) {
+      sm100::tc_fence_after();
+      const float inv = (a.splits == 1) ? 1.f / l_run : 1.f;
+      bf16 *o = a.O + ((size_t)max(my_slot, 0) * a.Hq + my_head) * HD;
+      const size_t pidx = ((size_t)sp * a.R + max(my_slot, 0)) * a.Hq + my_head;
+      float *po = a.part_O + pidx * HD;
 #pragma unroll
-        for (int d = 0; d < HD; d += 8) {
-          uint4 u;
-          __nv_bfloat162 h0 = __floats2bfloat162_rn(o_acc[d] * inv, o_acc[d + 1] * inv), h1 = __floats2bfloat162_rn(o_acc[d + 2] * inv, o_acc[d + 3] * inv),
-                         h2 = __floats2bfloat162_rn(o_acc[d + 4] * inv, o_acc[d + 5] * inv), h3 = __floats2bfloat162_rn(o_acc[d + 6] * inv, o_acc[d + 7] * inv);
-          u.x = *reinterpret_cast<uint32_t *>(&h0); u.y = *reinterpret_cast<uint32_t *>(&h1);
-          u.z = *reinterpret_cast<uint32_t *>(&h2); u.w = *reinterpret_cast<uint32_t *>(&h3);
-          *reinterpret_cast<uint4 *>(o + d) = u;
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t v[32];
+        if (nt > 0) { sm100::tmem_ld32(tmem_O + lane_addr + c * 32, v); sm100::tmem_wait_ld(); }
+        else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
-      } else {
-        const size_t idx = ((size_t)sp * a.R + my_slot) * a.Hq + my_head;
-        float *po = a.part_O + idx * HD;
+        if (my_slot >= 0) {
+          if (a.splits == 1) {
 #pragma unroll
-        for (int d = 0; d < HD; d += 4) *reinterpret_cast<float4 *>(po + d) = make_float4(o_acc[d], o_acc[d + 1], o_acc[d + 2], o_acc[d + 3]);
-        a.part_ml[idx * 2] = m_run; a.part_ml[idx * 2 + 1] = l_run;
+            for (int j = 0; j < 32; j += 8) {
+              uint4 u;
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv),
+                             h1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv),
+                             h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv),
+                             h3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
+              u.x = *reinterpret_cast<uint32_t *>(&h0); u.y = *reinterpret_cast<uint32_t *>(&h1);
+              u.z = *reinterpret_cast<uint32_t *>(&h2); u.w = *reinterpret_cast<uint32_t *>(&h3);
+              *reinterpret_cast<uint4 *>(o + c * 32 + j) = u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<uint4 *>(po + c * 32 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          }
+        }
       }
-    }
-    if (a.tile_stats && threadIdx.x == 64 && sp == 0 && kvh == 0) {
-      // a dense-mask kernel would visit every cached page up to the group's last position and
-      // every local row of the group for each query tile
-      atomicAdd(&a.tile_stats[0], (unsigned long long)nt_all);
+      if (my_slot >= 0 && a.splits > 1) { a.part_ml[pidx * 2] = m_ref; a.part_ml[pidx * 2 + 1] = l_run; }
     }
   }
 
   // ---- teardown ----
   sm100::tc_fence_before();
   __syncthreads();
-  if (abort_flag) {
+  if (ctl.abort_flag) {
     if (threadIdx.x == 0 && a.status) atomicExch(a.status, 2);
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     __syncthreads();

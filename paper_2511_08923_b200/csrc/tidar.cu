@@ -340,14 +340,14 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   a.tiles_per_group = (rows_per_group + a.spt - 1) / a.spt;
   a.n_groups = (R + rows_per_group - 1) / rows_per_group;
   const int units = a.n_groups * a.tiles_per_group * a.Hkv;
-  int splits = c->n_sms / std::max(units, 1);
+  int splits = 2 * c->n_sms / std::max(units, 1);          // two CTAs fit on an SM
   splits = std::min(splits, std::max(1, key_tiles_hint / 2));
   a.splits = std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
   a.seq = c->meta.seq; a.nvis = c->meta.nvis; a.loc0 = c->meta.loc0; a.nloc = c->meta.nloc;
   a.page_table = g.page_table; a.pages_per_seq = g.pages_per_seq;
   a.page_base_k = m.page_base_k; a.page_base_v = m.page_base_v;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)cf.head_dim);
-  a.O = O; a.part_O = c->attn_part_O; a.part_ml = c->attn_part_ml; a.tile_stats = nullptr; a.status = c->d_status;
+  a.O = O; a.part_O = c->attn_part_O; a.part_ml = c->attn_part_ml; a.status = c->d_status;
   const int grid = units * a.splits;
   {
     Launch l(c, TIDAR_TC_ATTN);
