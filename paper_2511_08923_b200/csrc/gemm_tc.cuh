@@ -45,8 +45,8 @@ struct Args {
   int stages;               // shared-memory ring depth
   int box_rows, n_box;      // activation rows per TMA box, boxes per stage
   int n1, n2;               // MMA N of the two instructions (n2 may be 0)
-  // MODE_SLAB: fp32 out[split][r][n]
-  float *out; long long slab_stride; int ldo;
+  // MODE_SLAB: out[split][r][n], fp32 or (slab_bf16) bf16; strides in elements
+  void *out; long long slab_stride; int ldo; int slab_bf16;
   // MODE_SWIGLU: weight rows interleave (gate f, up f); H[r][f] = silu(gate) * up, bf16
   bf16 *H; int ldh;
   // MODE_ARGMAX: per (CTA, lane quadrant) candidates, [gridDim*4][R] (index -1 = none; the caller
@@ -236,16 +236,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int n = tile * TILE_N + q * 32 + lane;       // this thread's output feature
       const int r_base = rb * g.rb_rows + c_begin;
       if (MODE == MODE_SLAB || !w.fused) {
-        // fp32 slab; columns are counted from the first tile of the split region
-        float *o = g.out + (long long)split * g.slab_stride + (n - g.tile_b0 * TILE_N);
+        // split-K partial sums; columns are counted from the first tile of the split region
+        const int nc = n - g.tile_b0 * TILE_N;
         const bool n_ok = n < g.N;
+        if (!g.slab_bf16) {
+          float *o = reinterpret_cast<float *>(g.out) + (long long)split * g.slab_stride + nc;
 #pragma unroll
-        for (int i = 0; i < 9; ++i) {
-          if (i * 16 < ncols) {
+          for (int i = 0; i < 9; ++i) {
+            if (i * 16 < ncols) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int r = r_base + i * 16 + j;
-              if (n_ok && r < g.R) o[(long long)r * g.ldo] = __uint_as_float(v[i][j]);
+              for (int j = 0; j < 16; ++j) {
+                const int r = r_base + i * 16 + j;
+                if (n_ok && r < g.R) o[(long long)r * g.ldo] = __uint_as_float(v[i][j]);
+              }
+            }
+          }
+        } else {
+          // bf16: lane pairs (2j, 2j+1) exchange so that the even lane stores features
+          // (n, n+1) of column c and the odd lane those of column c+1, 4 bytes each
+          bf16 *o = reinterpret_cast<bf16 *>(g.out) + (long long)split * g.slab_stride + (nc & ~1);
+          const bool odd = lane & 1;
+#pragma unroll
+          for (int i = 0; i < 9; ++i) {
+            if (i * 16 < ncols) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 2) {
+                const uint32_t send = odd ? v[i][j] : v[i][j + 1];
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                const float lo = __uint_as_float(odd ? recv : v[i][j]);          // feature n & ~1
+                const float hi = __uint_as_float(odd ? v[i][j + 1] : recv);      // feature n | 1
+                const int r = r_base + i * 16 + j + (odd ? 1 : 0);
+                if (n_ok && r < g.R) {
+                  __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+                  *reinterpret_cast<__nv_bfloat162 *>(o + (long long)r * g.ldo) = h2;
+                }
+              }
             }
           }
         }

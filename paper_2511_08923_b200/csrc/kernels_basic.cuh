@@ -3,6 +3,15 @@
 #pragma once
 #include "common.cuh"
 
+// Four consecutive split-K partial sums starting at p (fp32 or bf16 slabs).
+template <typename T> __device__ __forceinline__ float4 load4(const T *p);
+template <> __device__ __forceinline__ float4 load4<float>(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+template <> __device__ __forceinline__ float4 load4<bf16>(const bf16 *p) {
+  const uint2 u = *reinterpret_cast<const uint2 *>(p);
+  const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.x)), b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+
 // One embedding row (bf16, d a multiple of 8) -> fp32, 16-byte loads.
 __device__ __forceinline__ void embed_row_to_f32(const bf16 *__restrict__ e, float *__restrict__ x, int d) {
   for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
@@ -108,9 +117,9 @@ __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int R, int ha
 // partial results of the previous projection (fixed order: deterministic), then
 // A = bf16(X * rsqrt(mean(X^2) + eps) * gain).  One block per row.
 // ---------------------------------------------------------------------------
-template <int THREADS>
+template <int THREADS, typename SLAB>
 __global__ void __launch_bounds__(THREADS)
-rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials, int S, size_t partial_stride,
+rmsnorm_reduce_kernel(float *__restrict__ X, const SLAB *__restrict__ partials, int S, size_t partial_stride,
                       const bf16 *__restrict__ gain, float eps, int d, bf16 *__restrict__ A) {
   pdl_trigger();
   pdl_wait();
@@ -122,7 +131,7 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials,
   for (int c = threadIdx.x * 4; c < d; c += THREADS * 4) {
     float4 v = *reinterpret_cast<const float4 *>(xr + c);
     for (int s = 0; s < S; ++s) {
-      const float4 p = *reinterpret_cast<const float4 *>(partials + s * partial_stride + (size_t)r * d + c);
+      const float4 p = load4<SLAB>(partials + s * partial_stride + (size_t)r * d + c);
       v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
     }
     *reinterpret_cast<float4 *>(row + c) = v;
@@ -153,8 +162,9 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const float *__restrict__ partials,
 // (causal slots: kept if accepted, evicted otherwise; paper Section 3.3) or to the
 // step-local scratch (mask slots, never cached).  One block per row.
 // ---------------------------------------------------------------------------
+template <typename SLAB>
 __global__ void __launch_bounds__(256)
-rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
+rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
                RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
                bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
                bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
@@ -170,8 +180,8 @@ rope_kv_kernel(const float *__restrict__ partials, int S, size_t partial_stride,
     const size_t base = (size_t)r * N + (size_t)h * hd + i;
     float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;
     for (int s = 0; s < S; ++s) {
-      const float4 a = *reinterpret_cast<const float4 *>(partials + s * partial_stride + base);
-      const float4 b = *reinterpret_cast<const float4 *>(partials + s * partial_stride + base + half);
+      const float4 a = load4<SLAB>(partials + s * partial_stride + base);
+      const float4 b = load4<SLAB>(partials + s * partial_stride + base + half);
       x1.x += a.x; x1.y += a.y; x1.z += a.z; x1.w += a.w;
       x2.x += b.x; x2.y += b.y; x2.z += b.z; x2.w += b.w;
     }
@@ -210,21 +220,23 @@ __global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16
   H[t] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
 }
 
-// SwiGLU over fp32 split-K slabs [S][R][ld] whose columns interleave (gate, up) and cover
-// features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).
-__global__ void swiglu_slab_kernel(const float *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
+// SwiGLU over bf16 split-K slabs [S][R][ld] whose columns interleave (gate, up) and cover
+// features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).  Two features per thread.
+__global__ void swiglu_slab_kernel(const bf16 *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
                                    bf16 *__restrict__ H) {
   pdl_trigger();
   pdl_wait();
   const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= (size_t)R * nf) return;
-  const int r = (int)(t / nf), f = (int)(t % nf);
-  float g = 0.f, u = 0.f;
+  const int nf2 = nf / 2;
+  if (t >= (size_t)R * nf2) return;
+  const int r = (int)(t / nf2), f = (int)(t % nf2) * 2;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);                      // gate f, up f, gate f+1, up f+1
   for (int s = 0; s < S; ++s) {
-    const float2 v = *reinterpret_cast<const float2 *>(slabs + s * stride + (size_t)r * ld + 2 * f);
-    g += v.x; u += v.y;
+    const float4 v = load4<bf16>(slabs + s * stride + (size_t)r * ld + 2 * f);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
-  H[(size_t)r * ldh + f0 + f] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+  __nv_bfloat162 o = __floats2bfloat162_rn(acc.x / (1.f + __expf(-acc.x)) * acc.y, acc.z / (1.f + __expf(-acc.z)) * acc.w);
+  *reinterpret_cast<__nv_bfloat162 *>(H + (size_t)r * ldh + f0 + f) = o;
 }
 
 // Running per-row argmax over a chunk of logits [R][ncols] (fp32, leading dim ld)

@@ -244,7 +244,8 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   if (mode == gemm_tc::MODE_SLAB) {
     a.n_tiles_b = a.n_tiles;
     a.S = force_S > 0 ? std::min(force_S, a.kb_total) : gemm_tc::plan_splits(a.n_rb * a.n_tiles, a.kb_total, c->n_sms, c->S_max, 4);
-    a.out = slab_out ? slab_out : c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
+    a.out = slab_out ? (void *)slab_out : (void *)c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
+    a.slab_bf16 = slab_out ? 0 : 1;          // the step's slabs are bf16; an explicit output buffer gets exact fp32 slabs
   } else if (mode == gemm_tc::MODE_SWIGLU) {
     a.H = c->H; a.ldh = N / 2;
     a.fused_items = a.n_rb * a.n_tiles;
@@ -258,7 +259,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
       if (S2 >= 2 && (size_t)S2 * R * rem * gemm_tc::TILE_N <= c->partials_cap) {
         rem_tiles = rem;
         a.fused_items = full; a.tile_b0 = full; a.n_tiles_b = rem; a.S = S2;
-        a.out = c->partials; a.ldo = rem * gemm_tc::TILE_N; a.slab_stride = (long long)R * a.ldo;
+        a.out = c->partials; a.ldo = rem * gemm_tc::TILE_N; a.slab_stride = (long long)R * a.ldo; a.slab_bf16 = 1;
       }
     }
   } else {
@@ -279,7 +280,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
     const size_t n = (size_t)R * nf;
     c->launches++;
-    launch_pdl(swiglu_slab_kernel, (unsigned)((n + 255) / 256), 256, 0, c->stream, c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+    launch_pdl(swiglu_slab_kernel, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
                                                                            a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
   }
   if (S_out) *S_out = a.S;
@@ -377,10 +378,14 @@ void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *V
     attn_replay_kernel<64><<<grid, 32, 0, c->stream>>>(Q, Kp, Vp, g, c->meta, Kl, Vl, O, c->cfg.n_q_heads, scale);
 }
 
+// partials: split-K slabs of the previous projection, bf16 on the tensor-core path, fp32 on the replay path
 void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t stride, const bf16 *gain) {
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
-  launch_pdl(rmsnorm_reduce_kernel<512>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+  if (c->cfg.impl == 0)
+    launch_pdl(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+  else
+    launch_pdl(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
 }
 
 // The transformer stack over R assembled rows (metadata and X already filled).
@@ -407,7 +412,11 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
-      launch_pdl(rope_kv_kernel, R, 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+if (tc)
+        launch_pdl(rope_kv_kernel<bf16>, R, 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
+      else
+        launch_pdl(rope_kv_kernel<float>, R, 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     if (tc) {
@@ -841,7 +850,7 @@ int tidar_gemm(tidar_ctx *c, const void *A, const void *W, int32_t R, int32_t N,
     CUtensorMap tmW;
     if (gemm_tc::encode_2d(c->encode, &tmW, W, (uint64_t)N, (uint64_t)K, gemm_tc::TILE_N) != CUDA_SUCCESS)
       return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for W");
-    if (int rc = gemm_tc_launch(c, gemm_tc::MODE_SLAB, (const bf16 *)A, R, tmW, R, N, K, TIDAR_TC_GEMM, &S, &stride, nullptr, splits)) return rc;
+    if (int rc = gemm_tc_launch(c, gemm_tc::MODE_SLAB, (const bf16 *)A, R, tmW, R, N, K, TIDAR_TC_GEMM, &S, &stride, c->partials, splits)) return rc;
   } else {
     if (int rc = gemm_partials(c, (const bf16 *)A, R, (const bf16 *)W, nullptr, R, N, K, c->partials, &S, &stride, TIDAR_TC_GEMM)) return rc;
   }
