@@ -49,9 +49,9 @@ struct Args {
   void *out; long long slab_stride; int ldo; int slab_bf16;
   // MODE_SWIGLU: weight rows interleave (gate f, up f); H[r][f] = silu(gate) * up, bf16
   bf16 *H; int ldh;
-  // MODE_ARGMAX: per (CTA, lane quadrant) candidates, [gridDim*4][R] (index -1 = none; the caller
-  // pre-fills the index table with -1); optional fp32 dump [R][ld_dump]
-  float *cand_val; int32_t *cand_idx; float *dump; int ld_dump; int col0;
+  // MODE_ARGMAX: per (CTA, lane quadrant) candidates, [R][cand_ld >= gridDim*4] (index -1 = none; the
+  // caller pre-fills the index table with -1); optional fp32 dump [R][ld_dump]
+  float *cand_val; int32_t *cand_idx; int cand_ld; float *dump; int ld_dump; int col0;
   int *status;              // device word set to 1 when a bounded wait gave up
   __host__ __device__ int tile_b0_or_all() const { return n_tiles_b ? tile_b0 : n_tiles; }   // tiles per row block in the fused region
   __host__ __device__ int total_items() const { return fused_items + n_rb * n_tiles_b * S; }
@@ -212,7 +212,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int cidx = k * 32 + lane;
         const int r = cur_rb * g.rb_rows + c_begin + cidx;
         if (cidx < ncols && r < g.R) {
-          const long long o = (long long)(blockIdx.x * 4 + q) * g.R + r;
+          const long long o = (long long)r * g.cand_ld + (blockIdx.x * 4 + q);
           g.cand_val[o] = best_v[k]; g.cand_idx[o] = best_i[k] == 0x7fffffff ? -1 : best_i[k];
         }
         best_v[k] = -INFINITY; best_i[k] = 0x7fffffff;
@@ -296,31 +296,53 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
       } else {
         // Per column: best (value, index) over the 32 features of this warp, folded into a
-        // running best over all tiles this CTA processes (column c is kept by lane c % 32).
-        // Lowest index wins ties, NaN never wins.
+        // running best over all tiles this CTA processes.  The 32 lanes x 32 columns of a
+        // group are reduced by recursive halving: in the step with stride h a lane keeps the
+        // columns whose bit h equals its own lane bit h and hands the others to lane ^ h, so
+        // after five steps lane l holds the result of column 32*g + l (31 exchanges per 32
+        // columns instead of 160).  Lowest index wins ties, NaN never wins.
         if (rb != cur_rb) { flush_best(); cur_rb = rb; }
         const bool n_ok = n < g.N;
+        const int my_idx = (n_ok ? g.col0 + n : 0x7fffffff);
+        if (g.dump && n_ok) {
 #pragma unroll
-        for (int i = 0; i < 9; ++i) {
-          if (i * 16 < ncols) {
+          for (int i = 0; i < 9; ++i)
+            if (i * 16 < ncols) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int r = r_base + i * 16 + j;
-              float val = __uint_as_float(v[i][j]);
-              if (g.dump && n_ok && r < g.R) g.dump[(long long)r * g.ld_dump + n] = val;
-              int idx = g.col0 + n;
-              if (!n_ok || !(val == val)) { val = -INFINITY; idx = 0x7fffffff; }
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, val, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-                if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
-              }
-              const int cidx = i * 16 + j;
-              if (lane == (cidx & 31) && (val > best_v[cidx >> 5] || (val == best_v[cidx >> 5] && idx < best_i[cidx >> 5]))) {
-                best_v[cidx >> 5] = val; best_i[cidx >> 5] = idx;
+              for (int j = 0; j < 16; ++j) {
+                const int r = r_base + i * 16 + j;
+                if (r < g.R) g.dump[(long long)r * g.ld_dump + n] = __uint_as_float(v[i][j]);
               }
             }
+        }
+#pragma unroll
+        for (int grp = 0; grp < 5; ++grp) {
+          if (grp * 32 < ncols) {
+            float val[32]; int idx[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int i = grp * 2 + (j >> 4);
+              float x = (i < 9 && i * 16 < ncols) ? __uint_as_float(v[i < 9 ? i : 8][j & 15]) : -INFINITY;
+              const bool ok_v = n_ok && (x == x);
+              val[j] = ok_v ? x : -INFINITY; idx[j] = ok_v ? my_idx : 0x7fffffff;
+            }
+#pragma unroll
+            for (int h = 16; h >= 1; h >>= 1) {
+              const bool up = lane & h;
+#pragma unroll
+              for (int j = 0; j < h; ++j) {
+                // columns j (bit h clear) and j + h (bit h set) of the current, already folded, set
+                const float sv = up ? val[j] : val[j + h];
+                const int si = up ? idx[j] : idx[j + h];
+                const float ov = __shfl_xor_sync(0xffffffffu, sv, h);
+                const int oi = __shfl_xor_sync(0xffffffffu, si, h);
+                const float mv = up ? val[j + h] : val[j];
+                const int mi = up ? idx[j + h] : idx[j];
+                const bool take = ov > mv || (ov == mv && oi < mi);
+                val[j] = take ? ov : mv; idx[j] = take ? oi : mi;
+              }
+            }
+            if (val[0] > best_v[grp] || (val[0] == best_v[grp] && idx[0] < best_i[grp])) { best_v[grp] = val[0]; best_i[grp] = idx[0]; }
           }
         }
       }

@@ -272,34 +272,27 @@ __global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int nco
   }
 }
 
-// Final argmax over the candidates [G][R] produced by the fused LM-head epilogue (one
-// candidate per 32 vocabulary ids): one block per row; a candidate index of -1 means
+// Final argmax over the candidates [R][G] produced by the fused LM-head epilogue (one
+// candidate per CTA and lane quadrant): one warp per row; a candidate index of -1 means
 // "nothing valid".  Lowest index wins ties, which makes the result independent of the
 // order in which candidates are combined.
 __global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t *__restrict__ pi, int G, int R,
                                     float *__restrict__ best_val, int32_t *__restrict__ best_idx) {
   pdl_trigger();
   pdl_wait();
-  const int r = blockIdx.x;
+  const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (r >= R) return;
   float bv = -INFINITY; int bi = 0x7fffffff;
-  for (int g = threadIdx.x; g < G; g += blockDim.x) {
-    const float v = pv[(size_t)g * R + r]; const int i = pi[(size_t)g * R + r];
+  for (int g = lane; g < G; g += 32) {
+    const float v = pv[(size_t)r * G + g]; const int i = pi[(size_t)r * G + g];
     if (i >= 0 && (v > bv || (v == bv && i < bi))) { bv = v; bi = i; }
   }
-  __shared__ float sv[32]; __shared__ int si[32];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, bv, o); const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
     if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
   }
-  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
-      if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
-    if (bi == 0x7fffffff) bi = 0;
-    best_val[r] = bv; best_idx[r] = bi;
-  }
+  if (lane == 0) { best_val[r] = bv; best_idx[r] = bi == 0x7fffffff ? 0 : bi; }
 }
 
 // out[i] = sum over S slabs (fixed order) of in[s * stride + i].

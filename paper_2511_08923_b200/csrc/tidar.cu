@@ -264,7 +264,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     }
   } else {
     a.fused_items = a.n_rb * a.n_tiles;
-    a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.dump = c->dbg_logits; a.ld_dump = c->cfg.vocab; a.col0 = 0;
+    a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.cand_ld = c->n_sms * 4; a.dump = c->dbg_logits; a.ld_dump = c->cfg.vocab; a.col0 = 0;
   }
   a.status = c->d_status;
   const CUtensorMap *tmA = act_map(c, A, a_rows, K, a.box_rows);
@@ -446,7 +446,7 @@ if (tc)
     CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
     if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    launch_pdl(argmax_merge_kernel, R, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
+    launch_pdl(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
