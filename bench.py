@@ -229,6 +229,7 @@ def main():
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--per-l-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lib-debug", type=int, default=0, help="library debug bits (4: bf16 split-K partial sums; diagnostics, not the bench configuration)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -262,7 +263,7 @@ def main():
     stream = torch.cuda.Stream(device=dev)
     n_steps_total = args.warmup + 2 * args.steps + 8 + k * args.per_l_steps
     t = Tidar(sh, packed, k_max=k, max_batch=1, max_seq_len=n0 + (n_steps_total + 4) * k + 2 * k + 64, impl=impl,
-              device=dev, stream=stream)
+              device=dev, stream=stream, debug=args.lib_debug)
     prompt = gen_token_ids(sh.seed, tensor_id("prompt"), n0, sh.vocab - 1).numpy()
     t.prefill(0, prompt, k)
     sched = acceptance_schedule(SCHEDULE_SEED, args.warmup + 2 * args.steps, k).numpy()

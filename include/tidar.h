@@ -62,7 +62,10 @@ typedef struct {
                                last pass for the tidar_debug_get_* calls (costs memory:
                                rows*vocab*4 bytes); bit 1: overwrite evicted KV slots with
                                the largest finite bf16 after each step (any use of them
-                               with a non-zero weight would wreck the results)             */
+                               with a non-zero weight would wreck the results); bit 2:
+                               keep the split-K partial sums of the projections in bf16
+                               instead of fp32 (about 4 % faster, about 20 % more rounding
+                               noise in deep models; off by default)                      */
   int32_t impl;             /* 0: tensor-core kernels (tcgen05/TMEM/TMA);
                                1: plain fp32-accumulate CUDA-core kernels ("replay"), a
                                slow diagnostic path with the same data flow               */

@@ -220,9 +220,10 @@ __global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16
   H[t] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
 }
 
-// SwiGLU over bf16 split-K slabs [S][R][ld] whose columns interleave (gate, up) and cover
-// features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).  Two features per thread.
-__global__ void swiglu_slab_kernel(const bf16 *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
+// SwiGLU over split-K slabs [S][R][ld] (fp32 or bf16) whose columns interleave (gate, up) and
+// cover features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).  Two features per thread.
+template <typename SLAB>
+__global__ void swiglu_slab_kernel(const SLAB *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
                                    bf16 *__restrict__ H) {
   pdl_trigger();
   pdl_wait();
@@ -232,7 +233,7 @@ __global__ void swiglu_slab_kernel(const bf16 *__restrict__ slabs, int S, size_t
   const int r = (int)(t / nf2), f = (int)(t % nf2) * 2;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);                      // gate f, up f, gate f+1, up f+1
   for (int s = 0; s < S; ++s) {
-    const float4 v = load4<bf16>(slabs + s * stride + (size_t)r * ld + 2 * f);
+    const float4 v = load4<SLAB>(slabs + s * stride + (size_t)r * ld + 2 * f);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
   __nv_bfloat162 o = __floats2bfloat162_rn(acc.x / (1.f + __expf(-acc.x)) * acc.y, acc.z / (1.f + __expf(-acc.z)) * acc.w);

@@ -68,6 +68,7 @@ struct tidar_ctx {
   CUtensorMap tm_q, tm_kv, tm_kloc, tm_vloc;
   float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
+  bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
   float *cand_val = nullptr;
   int32_t *h_status = nullptr;
@@ -245,7 +246,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     a.n_tiles_b = a.n_tiles;
     a.S = force_S > 0 ? std::min(force_S, a.kb_total) : gemm_tc::plan_splits(a.n_rb * a.n_tiles, a.kb_total, c->n_sms, c->S_max, 4);
     a.out = slab_out ? (void *)slab_out : (void *)c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
-    a.slab_bf16 = slab_out ? 0 : 1;          // the step's slabs are bf16; an explicit output buffer gets exact fp32 slabs
+    a.slab_bf16 = (slab_out || !c->slab_bf16) ? 0 : 1;   // an explicit output buffer always gets exact fp32 slabs
   } else if (mode == gemm_tc::MODE_SWIGLU) {
     a.H = c->H; a.ldh = N / 2;
     a.fused_items = a.n_rb * a.n_tiles;
@@ -259,7 +260,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
       if (S2 >= 2 && (size_t)S2 * R * rem * gemm_tc::TILE_N <= c->partials_cap) {
         rem_tiles = rem;
         a.fused_items = full; a.tile_b0 = full; a.n_tiles_b = rem; a.S = S2;
-        a.out = c->partials; a.ldo = rem * gemm_tc::TILE_N; a.slab_stride = (long long)R * a.ldo; a.slab_bf16 = 1;
+        a.out = c->partials; a.ldo = rem * gemm_tc::TILE_N; a.slab_stride = (long long)R * a.ldo; a.slab_bf16 = c->slab_bf16 ? 1 : 0;
       }
     }
   } else {
@@ -280,7 +281,11 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
     const size_t n = (size_t)R * nf;
     c->launches++;
-    launch_pdl(swiglu_slab_kernel, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+    if (c->slab_bf16)
+      launch_pdl(swiglu_slab_kernel<bf16>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
+    else
+      launch_pdl(swiglu_slab_kernel<float>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const float *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
                                                                            a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
   }
   if (S_out) *S_out = a.S;
@@ -382,7 +387,7 @@ void launch_attention(tidar_ctx *c, const bf16 *Q, const bf16 *Kp, const bf16 *V
 void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t stride, const bf16 *gain) {
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
-  if (c->cfg.impl == 0)
+  if (c->cfg.impl == 0 && c->slab_bf16)
     launch_pdl(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
   else
     launch_pdl(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
@@ -412,7 +417,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
-if (tc)
+if (tc && c->slab_bf16)
         launch_pdl(rope_kv_kernel<bf16>, R, 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
       else
@@ -633,6 +638,7 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
   if ((uintptr_t)arena % 256) return fail(nullptr, TIDAR_EINVAL, "arena must be 256-byte aligned");
   tidar_ctx *c = new tidar_ctx;
   c->cfg = *cfg;
+  c->slab_bf16 = (cfg->debug & 4) != 0;
   c->stream = (cudaStream_t)cuda_stream;
   size_t need = 0;
   layout(*c, arena, &need);
