@@ -65,7 +65,9 @@ typedef struct {
                                with a non-zero weight would wreck the results); bit 2:
                                keep the split-K partial sums of the projections in bf16
                                instead of fp32 (about 4 % faster, about 20 % more rounding
-                               noise in deep models; off by default)                      */
+                               noise in deep models; off by default); bit 3: launch the
+                               kernels of a step one by one instead of replaying a captured
+                               graph (A/B diagnostics)                                    */
   int32_t impl;             /* 0: tensor-core kernels (tcgen05/TMEM/TMA);
                                1: plain fp32-accumulate CUDA-core kernels ("replay"), a
                                slow diagnostic path with the same data flow               */

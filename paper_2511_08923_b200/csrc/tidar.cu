@@ -68,6 +68,9 @@ struct tidar_ctx {
   CUtensorMap tm_q, tm_kv, tm_kloc, tm_vloc;
   float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
+  // the launches of one decode step as an executable graph, valid for one (k, n_seqs, attention split)
+  struct StepGraph { int k = 0, n_seqs = 0, splits = 0; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
+  bool graphs_ok = true;
   bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
   float *cand_val = nullptr;
@@ -333,6 +336,14 @@ bool encode_local_map(tidar_ctx *c, CUtensorMap *tm, const void *loc, long long 
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Key-range split of the attention kernel: fill the SMs (two CTAs fit on one) without
+// giving a CTA fewer than two key tiles.
+int attn_key_splits(const tidar_ctx *c, int units, int key_tiles_hint) {
+  int splits = 2 * c->n_sms / std::max(units, 1);
+  splits = std::min(splits, std::max(1, key_tiles_hint / 2));
+  return std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
+}
+
 struct AttnMaps { const CUtensorMap *q, *k, *v, *kloc, *vloc; int page_base_k, page_base_v; };
 
 // rows_per_group: slots per sequence (k(k+1) in a step; all rows in a first-pass chunk).
@@ -346,9 +357,7 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   a.tiles_per_group = (rows_per_group + a.spt - 1) / a.spt;
   a.n_groups = (R + rows_per_group - 1) / rows_per_group;
   const int units = a.n_groups * a.tiles_per_group * a.Hkv;
-  int splits = 2 * c->n_sms / std::max(units, 1);          // two CTAs fit on an SM
-  splits = std::min(splits, std::max(1, key_tiles_hint / 2));
-  a.splits = std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
+  a.splits = attn_key_splits(c, units, key_tiles_hint);
   a.seq = c->meta.seq; a.nvis = c->meta.nvis; a.loc0 = c->meta.loc0; a.nloc = c->meta.nloc;
   a.page_table = g.page_table; a.pages_per_seq = g.pages_per_seq;
   a.page_base_k = m.page_base_k; a.page_base_v = m.page_base_v;
@@ -541,6 +550,34 @@ int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
   return TIDAR_OK;
 }
 
+// Enqueues every operation of one decode step for the sequences staged in h_stage.
+int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint) {
+  const tidar_config &cf = c->cfg;
+  const int T = k * (k + 1), R = n_seqs * T;
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  {
+    Launch l(c, TIDAR_TC_EMBED);
+    launch_pdl(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
+               c->d_step_n, c->embed, cf.d_model, c->X);
+  }
+  if (int rc = forward_rows(c, R, true, T, key_tiles_hint)) return rc;
+  {
+    Launch l(c, TIDAR_TC_VERIFY);
+    launch_pdl(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
+               c->d_step_L, c->d_out);
+  }
+  {
+    Launch l(c, TIDAR_TC_VERIFY);
+    launch_pdl(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
+               (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
 int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced) {
   const tidar_config &cf = c->cfg;
   if (!seqs || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
@@ -564,30 +601,46 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   }
   const int T = k * (k + 1), R = n_seqs * T;
   for (int i = 0; i < n_seqs; ++i) { c->h_stage[i] = seqs[i]; c->h_stage[cf.max_batch + i] = forced ? forced[i] : 0; }
-  CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-  CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-  {
-    Launch l(c, TIDAR_TC_EMBED);
-    launch_pdl(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
-                                                   c->d_step_n, c->embed, cf.d_model, c->X);
-  }
   int min_n = 1 << 30;
   for (int i = 0; i < n_seqs; ++i) min_n = std::min(min_n, c->seqs[seqs[i]].n);
-  int rc = forward_rows(c, R, true, T, (min_n + k + 63) / 64);
-  if (rc) return rc;
-  {
-    Launch l(c, TIDAR_TC_VERIFY);
-    launch_pdl(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
-                                                       c->d_step_L, c->d_out);
+  const int hint = (min_n + k + 63) / 64;
+  // Every launch of a step has the same arguments from step to step (lengths, page tables and
+  // token blocks live in device memory), except for the attention key split, so the step is
+  // captured once per (k, n_seqs, split) and replayed.  Per-launch timing and the debug
+  // read-backs use plain launches.
+  bool launched = false;
+  if (cf.impl == 0 && c->graphs_ok && !c->timing && !(cf.debug & (1 | 8))) {
+    const int G = cf.n_q_heads / cf.n_kv_heads, spt = 128 / G;
+    const int splits = attn_key_splits(c, n_seqs * ((T + spt - 1) / spt) * cf.n_kv_heads, hint);
+    tidar_ctx::StepGraph &sg = c->sg;
+    if (!sg.exec || sg.k != k || sg.n_seqs != n_seqs || sg.splits != splits) {
+      if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
+      const int64_t l0 = c->launches;
+      cudaGraph_t graph = nullptr;
+      int rc = TIDAR_OK;
+      cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
+      if (e == cudaSuccess) {
+        rc = record_step(c, n_seqs, k, hint);
+        e = cudaStreamEndCapture(c->stream, &graph);
+      }
+      if (e == cudaSuccess && rc == TIDAR_OK && graph) e = cudaGraphInstantiate(&sg.exec, graph, 0);
+      if (graph) cudaGraphDestroy(graph);
+      if (e != cudaSuccess || rc != TIDAR_OK || !sg.exec) {
+        cudaGetLastError();                         // capture is not available here: plain launches from now on
+        sg.exec = nullptr; c->graphs_ok = false;
+      } else {
+        sg.k = k; sg.n_seqs = n_seqs; sg.splits = splits; sg.launches = c->launches - l0;
+      }
+      c->launches = l0;
+    }
+    if (sg.exec) {
+      CUDA_TRY(c, cudaGraphLaunch(sg.exec, c->stream));
+      c->launches += sg.launches;
+      launched = true;
+    }
   }
-  {
-    Launch l(c, TIDAR_TC_VERIFY);
-    launch_pdl(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
-                                                                       (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
-  }
-  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-  CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-  CUDA_TRY(c, cudaGetLastError());
+  if (!launched)
+    if (int rc = record_step(c, n_seqs, k, hint)) return rc;
   c->pending_seqs.assign(seqs, seqs + n_seqs);
   c->pending = true;
   c->last_rows = R; c->last_first_pos = -1;
@@ -741,6 +794,7 @@ int tidar_free(tidar_ctx *c) {
   if (!c) return TIDAR_EINVAL;
   cudaStreamSynchronize(c->stream);
   for (auto &t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+  if (c->sg.exec) cudaGraphExecDestroy(c->sg.exec);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
   return TIDAR_OK;
