@@ -234,7 +234,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     for (int i = 0; i < nt && ok; ++i) {
       const int t = t_begin + i;
       const int b = i & 1; const uint32_t bph = (uint32_t)(i >> 1) & 1u;
-      if (!sm100::mbar_wait(sm100::smem_u32(&ctl.s_full[b]), bph, abortp)) { ok = false; break; }
+      // a wait that gives up must take the whole warp out: the TMEM loads below are warp-collective
+      if (!__all_sync(0xffffffffu, sm100::mbar_wait(sm100::smem_u32(&ctl.s_full[b]), bph, abortp))) { ok = false; break; }
       sm100::tc_fence_after();
       uint32_t sv[64];
       {
@@ -284,7 +285,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       m_ref = m_new;
 
       // PV of the previous tile must be complete: it read P and updated O
-      if (!sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), ((uint32_t)i & 1u) ^ 1u, abortp)) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), ((uint32_t)i & 1u) ^ 1u, abortp))) { ok = false; break; }
       if (i > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         sm100::tc_fence_after();
 #pragma unroll
@@ -315,6 +316,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     // ---- output: O is complete once the last PV has finished ----
     if (ok && nt > 0) ok = sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), (uint32_t)(nt - 1) & 1u, abortp);
+    ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       sm100::tc_fence_after();
       const float inv = (a.splits == 1) ? 1.f / l_run : 1.f;
