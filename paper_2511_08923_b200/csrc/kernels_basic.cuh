@@ -160,7 +160,7 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const SLAB *__restrict__ partials, 
 // [S][R][(Hq+2Hkv)*hd].  Q heads are rotated and stored bf16 [R][Hq][hd]; K heads are
 // rotated, V heads copied; both go to the paged cache at the row's cache position
 // (causal slots: kept if accepted, evicted otherwise; paper Section 3.3) or to the
-// step-local scratch (mask slots, never cached).  One block per row.
+// step-local scratch (mask slots, never cached).  Grid (rows, unit chunks of 256).
 // ---------------------------------------------------------------------------
 template <typename SLAB>
 __global__ void __launch_bounds__(256)
@@ -170,12 +170,13 @@ rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, 
                bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
   pdl_trigger();
   pdl_wait();
-  // one block per row; a work unit is 4 consecutive dims i..i+3 of the first half of one
+  // a work unit is 4 consecutive dims i..i+3 of the first half of one
   // head together with their rotation partners i+hd/2..
   const int r = blockIdx.x, half = hd / 2, upr = half / 4;          // units per head
   const int H = Hq + 2 * Hkv, N = H * hd;
   const int cp = m.cache_pos[r], seq = m.seq[r], li = m.local_idx[r];
-  for (int u = threadIdx.x; u < H * upr; u += blockDim.x) {
+  // grid (rows, ceil(units / 256)): one unit per thread, so a row's latency is one round of loads
+  for (int u = blockIdx.y * blockDim.x + threadIdx.x; u < H * upr; u += gridDim.y * blockDim.x) {
     const int h = u / upr, i = (u % upr) * 4;
     const size_t base = (size_t)r * N + (size_t)h * hd + i;
     float4 x1 = make_float4(0.f, 0.f, 0.f, 0.f), x2 = x1;

@@ -426,11 +426,12 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     if ((rc = gemm_partials(c, c->A, RA, c->wqkv[l], tc ? &c->tm_wqkv[l] : nullptr, R, c->n_qkv, d, c->partials, &S, &stride, TIDAR_TC_GEMM))) return rc;
     {
       Launch ll(c, TIDAR_TC_ROPE);
+      const int rope_chunks = ((Hq + 2 * Hkv) * (hd / 8) + 255) / 256;
 if (tc && c->slab_bf16)
-        launch_pdl(rope_kv_kernel<bf16>, R, 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+        launch_pdl(rope_kv_kernel<bf16>, dim3(R, rope_chunks), 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
       else
-        launch_pdl(rope_kv_kernel<float>, R, 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+        launch_pdl(rope_kv_kernel<float>, dim3(R, rope_chunks), 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     if (tc) {
