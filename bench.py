@@ -352,12 +352,7 @@ def main():
               "hbm_frac_of_measured_peak": None}
 
     if world > 1:
-        tt = torch.tensor([ms_total, e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, e2e_s = float(tt[0]), float(tt[1])
-        tk = torch.tensor([tokens, tokens_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tokens, tokens_e2e = float(tk[0]), float(tk[1])
+        ms_total, e2e_s, tokens, tokens_e2e = aggregate_over_ranks(ms_total, e2e_s, tokens, tokens_e2e, dev)
 
     if rank == 0:
         pk, pk_src = peaks()
@@ -419,6 +414,18 @@ def main():
     t.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def aggregate_over_ranks(ms_total, e2e_s, tokens, tokens_e2e, device):
+    """Replicas only: every rank decodes its own sequence, nothing is exchanged on the data path.
+    The job's time is the slowest rank's (MAX), its tokens are all ranks' tokens (SUM).  The
+    process group is the caller's (NCCL under torchrun; gloo in the CPU test)."""
+    import torch.distributed as dist
+    tt = torch.tensor([ms_total, e2e_s], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    tk = torch.tensor([tokens, tokens_e2e], device=device, dtype=torch.float64)
+    dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+    return float(tt[0]), float(tt[1]), float(tk[0]), float(tk[1])
 
 
 DEFAULT_IMPL = 0
