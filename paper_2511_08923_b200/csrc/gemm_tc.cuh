@@ -14,7 +14,9 @@
 // loop over items.  Warp roles: warp 0 issues TMA loads into a ring of shared-memory
 // stages, warp 1 issues the MMAs into one fp32 accumulator in TMEM, warps 2..9 drain the
 // accumulator into registers (which frees it for the next item at once) and then run the
-// epilogue from registers while the next item's MMAs proceed.
+// epilogue from registers while the next item's MMAs proceed, and warp 10 watches the
+// stages' mbarriers on behalf of the MMA warp (which must not touch the memory pipeline
+// between its MMAs) and releases it through hardware barriers.
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -24,8 +26,8 @@ namespace gemm_tc {
 constexpr int TILE_N = 128;         // weight rows per tile (TMEM lanes)
 constexpr int TILE_K = 64;          // bf16 elements per 128-byte swizzled row
 constexpr int MAX_ROWS = 288;       // activation rows per row block (2 x 144 TMEM columns)
-constexpr int THREADS = 320;
 constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 32 * (3 + EPI_WARPS);   // TMA producer, MMA issuer, epilogue warps, stage watcher
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int SMEM_BUDGET = 220 * 1024;
 constexpr int TMEM_COLS = 512;
@@ -147,27 +149,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    // One thread issues every MMA, so its instruction count per K block bounds the whole
-    // kernel: descriptors are built once and advanced with plain adds (the start-address
+    // One thread issues every MMA, and it issues them barely faster than the tensor pipe
+    // retires them, so nothing else may sit in its instruction stream: a test of an mbarrier
+    // (any access through the memory pipeline) completes only once the MMAs queued before it
+    // have gone out, and the pipe runs dry for ~250 cycles per K block.  The watcher warp
+    // therefore does the mbarrier waits and releases this warp through one hardware barrier
+    // per stage.  Descriptors are built once and advanced with plain adds (the start-address
     // field counts 16-byte units and never carries out of its 14 bits inside shared memory).
-    if (lane == 0) {
-      const uint32_t idesc1 = sm100::make_idesc_bf16(TILE_N, g.n1), idesc2 = sm100::make_idesc_bf16(TILE_N, g.n2 ? g.n2 : 16);
-      const uint64_t desc0 = sm100::make_desc_sw128(smem0);             // stage 0 weights
-      const uint64_t stage16 = (uint64_t)(stage_bytes >> 4);
-      const uint64_t a_off16 = (uint64_t)(W_STAGE_BYTES >> 4), a2_off16 = (uint64_t)(g.n1 * 8);
-      const uint32_t tmem_acc2 = tmem_acc + (uint32_t)g.n1;
-      const bool two = g.n2 != 0;
-      int s = 0; uint32_t ph = 0; bool ok = true; uint32_t it = 0;
-      uint64_t wd = desc0;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-        const Item w = decode_item(g, item);
-        const int kb0 = w.kb0, kb1 = w.kb1;
-        if (!sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp)) { ok = false; break; }
+    //
+    // This warp and the watcher run the same (item, K block) schedule to the end whatever
+    // happens elsewhere, one barrier operation each per K block, so neither can be left
+    // waiting for the other; after a failed wait the MMAs read stale tiles, which is harmless,
+    // and the status word reports the failure.
+    const uint32_t idesc1 = sm100::make_idesc_bf16(TILE_N, g.n1), idesc2 = sm100::make_idesc_bf16(TILE_N, g.n2 ? g.n2 : 16);
+    const uint64_t desc0 = sm100::make_desc_sw128(smem0);             // stage 0 weights
+    const uint64_t stage16 = (uint64_t)(stage_bytes >> 4);
+    const uint64_t a_off16 = (uint64_t)(W_STAGE_BYTES >> 4), a2_off16 = (uint64_t)(g.n1 * 8);
+    const uint32_t tmem_acc2 = tmem_acc + (uint32_t)g.n1;
+    const bool two = g.n2 != 0;
+    int s = 0;
+    uint64_t wd = desc0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const Item w = decode_item(g, item);
+      const int kb0 = w.kb0, kb1 = w.kb1;
+      uint32_t acc = 0u;                 // the watcher's first release of an item also says that the accumulator is free
+      for (int kb = kb0; kb < kb1; ++kb) {
+        sm100::named_bar_sync(1u + (uint32_t)s, 64);
         sm100::tc_fence_after();
-        uint32_t acc = 0u;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!sm100::mbar_wait(sm100::smem_u32(&full_bar[s]), ph, abortp)) { ok = false; break; }
-          sm100::tc_fence_after();
+        if (lane == 0) {
           const uint64_t ad = wd + a_off16;
           if (two) {
             const uint64_t ad2 = ad + a2_off16;
@@ -185,10 +194,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             }
           }
           sm100::mma_commit(sm100::smem_u32(&empty_bar[s]));     // stage reusable once these MMAs have read it
-          wd += stage16;
-          if (++s == g.stages) { s = 0; ph ^= 1u; wd = desc0; }
         }
-        if (ok) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
+        __syncwarp();
+        wd += stage16;
+        if (++s == g.stages) { s = 0; wd = desc0; }
+      }
+      if (lane == 0) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
+      __syncwarp();
+    }
+  } else if (warp == 2 + EPI_WARPS) {
+    // ===================== stage watcher =====================
+    // Waits (bounded) for the accumulator to be drained and for each stage's loads to land,
+    // then arrives on the stage's hardware barrier.  A stage's barrier cannot be arrived on
+    // twice before the MMA warp has passed it: the second landing needs the producer's refill,
+    // which needs the MMA warp's commit for the first.  After a failed wait that argument no
+    // longer holds, so from then on the watcher meets the MMA warp at every barrier instead.
+    int s = 0; uint32_t ph = 0, it = 0; bool failed = false;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+      const Item w = decode_item(g, item);
+      if (!failed) {
+        bool ok = true;
+        if (lane == 0) ok = sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp);
+        failed = !__shfl_sync(0xffffffffu, ok, 0);
+      }
+      for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        if (!failed) {
+          bool ok = true;
+          if (lane == 0) ok = sm100::mbar_wait(sm100::smem_u32(&full_bar[s]), ph, abortp);
+          failed = !__shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (!failed) sm100::named_bar_arrive(1u + (uint32_t)s, 64);
+        else sm100::named_bar_sync(1u + (uint32_t)s, 64);
+        if (++s == g.stages) { s = 0; ph ^= 1u; }
       }
     }
   } else {

@@ -50,6 +50,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// ---- named barriers (hardware barriers 1..15 of the CTA; 0 is __syncthreads) -------------
+// Both are executed by whole, converged warps; `threads` counts every participating thread
+// (arriving and waiting) and is a multiple of 32.  Unlike an mbarrier test, waiting here does
+// not go through the memory pipeline, so a warp that issues tcgen05.mma can wait on it without
+// its queued MMAs draining first.
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // ---- TMA ----------------------------------------------------------------------
 __device__ __forceinline__ uint64_t policy_evict_first() {
   uint64_t p;
