@@ -73,7 +73,9 @@ __device__ __forceinline__ Item decode_item(const Args &g, int item) {
   return w;
 }
 
-__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
+// silu(g) * u.  The fast division is exact enough for a bf16 result (2 ulp of fp32) and returns
+// the right limit (-0) when exp(-g) overflows.
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
 
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -82,6 +84,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], tmem_full_bar, tmem_empty_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  __shared__ __align__(16) uint16_t epi_stage[MODE == MODE_SWIGLU ? EPI_WARPS : 1][16][16];   // MODE_SWIGLU: one 16-column chunk per epilogue warp, [column][feature]
 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -312,23 +315,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
         }
       } else if (MODE == MODE_SWIGLU) {
-        // lane pairs (2j, 2j+1) hold gate and up of feature n/2; the even lane finishes
-        // column c, the odd lane column c+1, after one exchange per column pair.
-        const int f = n >> 1;
-        const bool f_ok = n < g.N;
+        // Lane pairs (2j, 2j+1) hold gate and up of feature n/2; the even lane finishes
+        // column c, the odd lane column c+1, after one exchange per column pair.  The
+        // results of a 16-column chunk (16 columns x 16 features per warp) are turned
+        // through shared memory so that every lane stores 8 consecutive features of one
+        // row with one 16-byte store: 2-byte stores from each lane took 18 us per tile.
         const bool odd = lane & 1;
+        uint16_t (*stage)[16] = epi_stage[warp - 2];
+        const int srow = lane >> 1, sf = (lane & 1) * 8;
+        const int f0 = ((tile * TILE_N + q * 32) >> 1) + sf;          // first of this lane's 8 features
+        const int n_feat = g.N >> 1;
 #pragma unroll
         for (int i = 0; i < 9; ++i) {
           if (i * 16 < ncols) {
+            // exchanges first, then eight independent silu chains: one chain at a time is
+            // bound by instruction latency (16 us per tile instead of 2)
+            uint32_t recv[8];
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-              const uint32_t send = odd ? v[i][j] : v[i][j + 1];
-              const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-              const float gate = __uint_as_float(odd ? recv : v[i][j]);
-              const float up = __uint_as_float(odd ? v[i][j + 1] : recv);
-              const int r = r_base + i * 16 + j + (odd ? 1 : 0);
-              if (f_ok && r < g.R) g.H[(long long)r * g.ldh + f] = __float2bfloat16(silu_mul(gate, up));
+            for (int j = 0; j < 8; ++j) recv[j] = __shfl_xor_sync(0xffffffffu, odd ? v[i][2 * j] : v[i][2 * j + 1], 1);
+            float h[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float gate = __uint_as_float(odd ? recv[j] : v[i][2 * j]);
+              const float up = __uint_as_float(odd ? v[i][2 * j + 1] : recv[j]);
+              h[j] = silu_mul(gate, up);
             }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) stage[2 * j + (odd ? 1 : 0)][lane >> 1] = __bfloat16_as_ushort(__float2bfloat16(h[j]));
+            __syncwarp();
+            const uint4 packed = *reinterpret_cast<const uint4 *>(&stage[srow][sf]);
+            const int r = r_base + i * 16 + srow;
+            if (r < g.R) {
+              bf16 *dst = g.H + (long long)r * g.ldh + f0;
+              if (f0 + 8 <= n_feat && (g.ldh & 7) == 0) {
+                *reinterpret_cast<uint4 *>(dst) = packed;
+              } else {
+                const uint16_t *e = reinterpret_cast<const uint16_t *>(&packed);
+                for (int t = 0; t < 8; ++t)
+                  if (f0 + t < n_feat) dst[t] = __ushort_as_bfloat16(e[t]);
+              }
+            }
+            __syncwarp();
           }
         }
       } else {
@@ -421,8 +448,8 @@ inline CUresult encode_2d(EncodeTiledFn fn, CUtensorMap *tm, const void *base, u
 }
 
 // Row-block geometry for R activation rows.
-inline void plan_rows(int R, Args &a) {
-  a.n_rb = (R + MAX_ROWS - 1) / MAX_ROWS;
+inline void plan_rows(int R, Args &a, int max_rows = MAX_ROWS) {
+  a.n_rb = (R + max_rows - 1) / max_rows;
   const int per = (R + a.n_rb - 1) / a.n_rb;
   a.rb_rows = (per + 15) / 16 * 16;
   if (a.rb_rows <= 256) { a.box_rows = a.rb_rows; a.n_box = 1; a.n1 = a.rb_rows; a.n2 = 0; }
