@@ -11,8 +11,11 @@
 // of up to 144 columns), so no tensor-core work is wasted on padding rows.
 //
 // Work item = (row block, 128-row weight tile, K split).  Persistent CTAs, one per SM,
-// loop over items.  Warp roles: warp 0 issues TMA loads into a ring of shared-memory
-// stages, warp 1 issues the MMAs into one fp32 accumulator in TMEM, warps 2..9 drain the
+// loop over items.  Warp roles: warp 0 streams weight tiles and warp 11 activation tiles by
+// TMA into two rings of shared-memory stages (the weight ring is the deep one: a tile comes
+// from HBM, takes > 1 us to arrive and is what bounds the kernel, while the wide activation
+// tile comes from L2 and only needs to be a little ahead), warp 1 issues the MMAs into one
+// fp32 accumulator in TMEM, warps 2..9 drain the
 // accumulator into registers (which frees it for the next item at once) and then run the
 // epilogue from registers while the next item's MMAs proceed, and warp 10 watches the
 // stages' mbarriers on behalf of the MMA warp (which must not touch the memory pipeline
@@ -27,7 +30,7 @@ constexpr int TILE_N = 128;         // weight rows per tile (TMEM lanes)
 constexpr int TILE_K = 64;          // bf16 elements per 128-byte swizzled row
 constexpr int MAX_ROWS = 288;       // activation rows per row block (2 x 144 TMEM columns)
 constexpr int EPI_WARPS = 8;
-constexpr int THREADS = 32 * (3 + EPI_WARPS);   // TMA producer, MMA issuer, epilogue warps, stage watcher
+constexpr int THREADS = 32 * (4 + EPI_WARPS);   // weight producer, MMA issuer, epilogue warps, stage watcher, activation producer
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int SMEM_BUDGET = 220 * 1024;
 constexpr int TMEM_COLS = 512;
@@ -44,7 +47,7 @@ struct Args {
                             // the rest are tiles tile_b0.. split S ways along K, written as fp32 slabs
   int tile_b0, n_tiles_b;   // first tile and tile count of the split region
   int kb_total;             // K / 64
-  int stages;               // shared-memory ring depth
+  int w_stages, a_stages;   // depths of the weight ring (<= 8) and of the activation ring (<= w_stages)
   int box_rows, n_box;      // activation rows per TMA box, boxes per stage
   int n1, n2;               // MMA N of the two instructions (n2 may be 0)
   // MODE_SLAB: out[split][r][n], fp32 or (slab_bf16) bf16; strides in elements
@@ -81,7 +84,7 @@ template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], tmem_full_bar, tmem_empty_bar;
+  __shared__ __align__(8) uint64_t w_full[8], w_empty[8], a_full[8], a_empty[8], tmem_full_bar, tmem_empty_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   __shared__ __align__(16) uint16_t epi_stage[MODE == MODE_SWIGLU ? EPI_WARPS : 1][16][16];   // MODE_SWIGLU: one 16-column chunk per epilogue warp, [column][feature]
@@ -89,13 +92,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem0 = (sm100::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const int a_stage_bytes = g.rb_rows * TILE_K * 2;
-  const int stage_bytes = W_STAGE_BYTES + a_stage_bytes;            // multiple of 1024 (rb_rows % 16 == 0)
+  const int a_stage_bytes = g.rb_rows * TILE_K * 2;                 // multiple of 1024 (rb_rows % 16 == 0)
+  const uint32_t smem_a0 = smem0 + (uint32_t)g.w_stages * W_STAGE_BYTES;   // activation ring behind the weight ring
   const int n_items = g.total_items();
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < g.stages; ++s) { sm100::mbar_init(sm100::smem_u32(&full_bar[s]), 1); sm100::mbar_init(sm100::smem_u32(&empty_bar[s]), 1); }
+    for (int s = 0; s < 8; ++s) {
+      sm100::mbar_init(sm100::smem_u32(&w_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&w_empty[s]), 1);
+      sm100::mbar_init(sm100::smem_u32(&a_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&a_empty[s]), 1);
+    }
     sm100::mbar_init(sm100::smem_u32(&tmem_full_bar), 1);
     sm100::mbar_init(sm100::smem_u32(&tmem_empty_bar), EPI_WARPS);
     sm100::fence_mbar_init();
@@ -112,41 +118,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   volatile int *abortp = &abort_flag;
 
   if (warp == 0) {
-    // ===================== TMA producer =====================
+    // ===================== weight producer =====================
     if (lane == 0) {
       sm100::prefetch_tensormap(&tmW);
-      sm100::prefetch_tensormap(&tmA);
-      const uint64_t pol_w = sm100::policy_evict_first(), pol_a = sm100::policy_evict_last();
+      const uint64_t pol_w = sm100::policy_evict_first();
       int s = 0; uint32_t ph = 0; bool ok = true;
-      // Weights are never written by a kernel, so the first stages' weight tiles are requested
-      // before waiting for the previous kernel; their activation tiles follow the wait.
-      int pre = 0;
-      if ((int)blockIdx.x < n_items) {
-        const Item w0 = decode_item(g, blockIdx.x);
-        pre = min(g.stages, w0.kb1 - w0.kb0);
-        for (int i = 0; i < pre; ++i) {
-          const uint32_t fb = sm100::smem_u32(&full_bar[i]);
-          sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
-          sm100::tma_load_2d(smem0 + (uint32_t)i * stage_bytes, &tmW, fb, (w0.kb0 + i) * TILE_K, w0.tile * TILE_N, pol_w);
-        }
-      }
-      pdl_wait();
+      // Weights are never written by a kernel, so nothing here waits for the previous kernel:
+      // the ring fills while that kernel is still finishing.
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item w = decode_item(g, item);
-        const int tile = w.tile, rb = w.rb;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
-          const uint32_t fb = sm100::smem_u32(&full_bar[s]);
-          const uint32_t sw = smem0 + (uint32_t)s * stage_bytes, sa = sw + W_STAGE_BYTES;
-          if (pre > 0) {
-            --pre;                                   // weights of this stage are already on their way
-          } else {
-            if (!sm100::mbar_wait(sm100::smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) { ok = false; break; }
-            sm100::mbar_expect_tx(fb, (uint32_t)stage_bytes);
-            sm100::tma_load_2d(sw, &tmW, fb, kb * TILE_K, tile * TILE_N, pol_w);
-          }
+          if (!sm100::mbar_wait(sm100::smem_u32(&w_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+          const uint32_t fb = sm100::smem_u32(&w_full[s]);
+          sm100::mbar_expect_tx(fb, (uint32_t)W_STAGE_BYTES);
+          sm100::tma_load_2d(smem0 + (uint32_t)s * W_STAGE_BYTES, &tmW, fb, kb * TILE_K, w.tile * TILE_N, pol_w);
+          if (++s == g.w_stages) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 3 + EPI_WARPS) {
+    // ===================== activation producer =====================
+    if (lane == 0) {
+      sm100::prefetch_tensormap(&tmA);
+      const uint64_t pol_a = sm100::policy_evict_last();
+      int s = 0; uint32_t ph = 0; bool ok = true;
+      pdl_wait();                      // the activations are the previous kernel's output
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const Item w = decode_item(g, item);
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+          if (!sm100::mbar_wait(sm100::smem_u32(&a_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
+          const uint32_t fb = sm100::smem_u32(&a_full[s]);
+          const uint32_t sa = smem_a0 + (uint32_t)s * a_stage_bytes;
+          sm100::mbar_expect_tx(fb, (uint32_t)a_stage_bytes);
           for (int b = 0; b < g.n_box; ++b)
-            sm100::tma_load_2d(sa + (uint32_t)(b * g.box_rows * TILE_K * 2), &tmA, fb, kb * TILE_K, rb * g.rb_rows + b * g.box_rows, pol_a);
-          if (++s == g.stages) { s = 0; ph ^= 1u; }
+            sm100::tma_load_2d(sa + (uint32_t)(b * g.box_rows * TILE_K * 2), &tmA, fb, kb * TILE_K, w.rb * g.rb_rows + b * g.box_rows, pol_a);
+          if (++s == g.a_stages) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -165,13 +171,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // waiting for the other; after a failed wait the MMAs read stale tiles, which is harmless,
     // and the status word reports the failure.
     const uint32_t idesc1 = sm100::make_idesc_bf16(TILE_N, g.n1), idesc2 = sm100::make_idesc_bf16(TILE_N, g.n2 ? g.n2 : 16);
-    const uint64_t desc0 = sm100::make_desc_sw128(smem0);             // stage 0 weights
-    const uint64_t stage16 = (uint64_t)(stage_bytes >> 4);
-    const uint64_t a_off16 = (uint64_t)(W_STAGE_BYTES >> 4), a2_off16 = (uint64_t)(g.n1 * 8);
+    const uint64_t wdesc0 = sm100::make_desc_sw128(smem0), adesc0 = sm100::make_desc_sw128(smem_a0);   // stage 0 of each ring
+    const uint64_t wstage16 = (uint64_t)(W_STAGE_BYTES >> 4), astage16 = (uint64_t)(a_stage_bytes >> 4);
+    const uint64_t a2_off16 = (uint64_t)(g.n1 * 8);
     const uint32_t tmem_acc2 = tmem_acc + (uint32_t)g.n1;
     const bool two = g.n2 != 0;
-    int s = 0;
-    uint64_t wd = desc0;
+    int s = 0, sa = 0;
+    uint64_t wd = wdesc0, ad = adesc0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
       const Item w = decode_item(g, item);
       const int kb0 = w.kb0, kb1 = w.kb1;
@@ -180,7 +186,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         sm100::named_bar_sync(1u + (uint32_t)s, 64);
         sm100::tc_fence_after();
         if (lane == 0) {
-          const uint64_t ad = wd + a_off16;
           if (two) {
             const uint64_t ad2 = ad + a2_off16;
 #pragma unroll
@@ -196,11 +201,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
               acc = 1u;
             }
           }
-          sm100::mma_commit(sm100::smem_u32(&empty_bar[s]));     // stage reusable once these MMAs have read it
+          sm100::mma_commit(sm100::smem_u32(&w_empty[s]));       // both stages reusable once these MMAs have read them
+          sm100::mma_commit(sm100::smem_u32(&a_empty[sa]));
         }
         __syncwarp();
-        wd += stage16;
-        if (++s == g.stages) { s = 0; wd = desc0; }
+        wd += wstage16; ad += astage16;
+        if (++s == g.w_stages) { s = 0; wd = wdesc0; }
+        if (++sa == g.a_stages) { sa = 0; ad = adesc0; }
       }
       if (lane == 0) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
       __syncwarp();
@@ -212,7 +219,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // twice before the MMA warp has passed it: the second landing needs the producer's refill,
     // which needs the MMA warp's commit for the first.  After a failed wait that argument no
     // longer holds, so from then on the watcher meets the MMA warp at every barrier instead.
-    int s = 0; uint32_t ph = 0, it = 0; bool failed = false;
+    int s = 0, sa = 0; uint32_t ph = 0, pha = 0, it = 0; bool failed = false;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
       const Item w = decode_item(g, item);
       if (!failed) {
@@ -223,15 +230,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int kb = w.kb0; kb < w.kb1; ++kb) {
         if (!failed) {
           bool ok = true;
-          if (lane == 0) ok = sm100::mbar_wait(sm100::smem_u32(&full_bar[s]), ph, abortp);
+          if (lane == 0) ok = sm100::mbar_wait(sm100::smem_u32(&w_full[s]), ph, abortp) && sm100::mbar_wait(sm100::smem_u32(&a_full[sa]), pha, abortp);
           failed = !__shfl_sync(0xffffffffu, ok, 0);
         }
         if (!failed) sm100::named_bar_arrive(1u + (uint32_t)s, 64);
         else sm100::named_bar_sync(1u + (uint32_t)s, 64);
-        if (++s == g.stages) { s = 0; ph ^= 1u; }
+        if (++s == g.w_stages) { s = 0; ph ^= 1u; }
+        if (++sa == g.a_stages) { sa = 0; pha ^= 1u; }
       }
     }
-  } else {
+  } else if (warp >= 2 && warp < 2 + EPI_WARPS) {
     // ===================== epilogue =====================
     pdl_wait();
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
@@ -454,11 +462,16 @@ inline void plan_rows(int R, Args &a, int max_rows = MAX_ROWS) {
   a.rb_rows = (per + 15) / 16 * 16;
   if (a.rb_rows <= 256) { a.box_rows = a.rb_rows; a.n_box = 1; a.n1 = a.rb_rows; a.n2 = 0; }
   else { a.box_rows = a.rb_rows / 2; a.n_box = 2; a.n1 = ((a.rb_rows / 2 + 15) / 16) * 16; a.n2 = a.rb_rows - a.n1; }
-  const int stage = W_STAGE_BYTES + a.rb_rows * TILE_K * 2;
-  a.stages = SMEM_BUDGET / stage;
-  if (a.stages > 8) a.stages = 8;
+  // Three activation stages keep that ring a K block ahead of the MMAs; the weight ring gets
+  // the rest of the budget.  Small row blocks get equally deep rings.
+  const int a_stage = a.rb_rows * TILE_K * 2;
+  a.a_stages = 3;
+  a.w_stages = (SMEM_BUDGET - a.a_stages * a_stage) / W_STAGE_BYTES;
+  if (a.w_stages > 8) a.w_stages = 8;
+  if (a.w_stages < 3) a.w_stages = 3;
+  while (a.a_stages < a.w_stages && (a.a_stages + 1) * a_stage + a.w_stages * W_STAGE_BYTES <= SMEM_BUDGET) a.a_stages++;
 }
-inline size_t smem_bytes(const Args &a) { return (size_t)a.stages * (W_STAGE_BYTES + a.rb_rows * TILE_K * 2) + 1024; }
+inline size_t smem_bytes(const Args &a) { return (size_t)a.w_stages * W_STAGE_BYTES + (size_t)a.a_stages * (a.rb_rows * TILE_K * 2) + 1024; }
 
 // K splits: fill the SMs with whole waves of equally sized items, keeping at least
 // min_kb K blocks per item.
