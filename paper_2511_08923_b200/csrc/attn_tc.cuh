@@ -259,28 +259,42 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           lo = max(0, my_loc0 - base); hi = my_nloc > 0 ? min(KT, my_loc0 + my_nloc - base) : 0;
         }
       }
-      float mx = -INFINITY;
+      // Softmax of the tile in base 2.  The scores stay raw in sv: the scale is applied inside
+      // one FMA per element (s * scale - m), masking is skipped for tiles that are visible in
+      // full (all cached keys but the last tile of a row), and the max and the sum run as
+      // four independent chains: this loop, not the MMAs, bounds the kernel.
+      if (lo > 0 || hi < KT) {
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        float s = __uint_as_float(sv[j]) * a.scale_log2;
-        s = (j >= lo && j < hi) ? s : -INFINITY;
-        sv[j] = __float_as_uint(s);
-        mx = fmaxf(mx, s);
+        for (int j = 0; j < 64; ++j)
+          if (j < lo || j >= hi) sv[j] = 0xff800000u;          // -inf
       }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < 64; j += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sv[j + u]));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;     // scale > 0; -inf stays -inf
       // raise the reference only when this tile exceeds it by more than the threshold
       // (-inf + threshold = -inf, so the first visible key always sets it)
       const float m_new = (mx > m_ref + RAISE_THRESHOLD) ? mx : m_ref;
       const float alpha = (m_new == m_ref) ? 1.f : exp2f(m_ref - m_new);      // m_ref = -inf gives 0
-      const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-      float sum = 0.f;
+      const float neg_m = (m_new == -INFINITY) ? 0.f : -m_new;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
-      for (int j = 0; j < 64; j += 2) {
-        const float p0 = exp2f(__uint_as_float(sv[j]) - m_safe), p1 = exp2f(__uint_as_float(sv[j + 1]) - m_safe);
-        sum += p0 + p1;
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-        pk[j >> 1] = *reinterpret_cast<uint32_t *>(&h2);
+      for (int j = 0; j < 64; j += 4) {
+        float p[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          p[u] = sm100::ex2_approx(fmaf(__uint_as_float(sv[j + u]), a.scale_log2, neg_m));   // -inf -> 0
+          sum4[u] += p[u];
+        }
+        __nv_bfloat162 h01 = __floats2bfloat162_rn(p[0], p[1]), h23 = __floats2bfloat162_rn(p[2], p[3]);
+        pk[j >> 1] = *reinterpret_cast<uint32_t *>(&h01);
+        pk[(j >> 1) + 1] = *reinterpret_cast<uint32_t *>(&h23);
       }
+      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l_run = l_run * alpha + sum;
       m_ref = m_new;
 

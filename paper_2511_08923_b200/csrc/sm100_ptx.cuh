@@ -50,6 +50,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// 2^x on the special-function unit, one instruction (denormal results flush to zero;
+// 2^-inf = 0, relative error about 2^-22).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ---- named barriers (hardware barriers 1..15 of the CTA; 0 is __syncthreads) -------------
 // Both are executed by whole, converged warps; `threads` counts every participating thread
 // (arriving and waiting) and is a multiple of 32.  Unlike an mbarrier test, waiting here does
