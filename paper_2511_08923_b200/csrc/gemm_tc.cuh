@@ -11,13 +11,13 @@
 // of up to 144 columns), so no tensor-core work is wasted on padding rows.
 //
 // Work item = (row block, 128-row weight tile, K split).  Persistent CTAs, one per SM,
-// loop over items.  Warp roles: warp 0 streams weight tiles and warp 11 activation tiles by
+// loop over items.  Warp roles: warp 0 streams weight tiles and warp 3 activation tiles by
 // TMA into two rings of shared-memory stages (the weight ring is the deep one: a tile comes
 // from HBM, takes > 1 us to arrive and is what bounds the kernel, while the wide activation
 // tile comes from L2 and only needs to be a little ahead), warp 1 issues the MMAs into one
-// fp32 accumulator in TMEM, warps 2..9 drain the
+// fp32 accumulator in TMEM, warps 4..11 drain the
 // accumulator into registers (which frees it for the next item at once) and then run the
-// epilogue from registers while the next item's MMAs proceed, and warp 10 watches the
+// epilogue from registers while the next item's MMAs proceed, and warp 2 watches the
 // stages' mbarriers on behalf of the MMA warp (which must not touch the memory pipeline
 // between its MMAs) and releases it through hardware barriers.
 #pragma once
@@ -30,7 +30,9 @@ constexpr int TILE_N = 128;         // weight rows per tile (TMEM lanes)
 constexpr int TILE_K = 64;          // bf16 elements per 128-byte swizzled row
 constexpr int MAX_ROWS = 288;       // activation rows per row block (2 x 144 TMEM columns)
 constexpr int EPI_WARPS = 8;
-constexpr int THREADS = 32 * (4 + EPI_WARPS);   // weight producer, MMA issuer, epilogue warps, stage watcher, activation producer
+constexpr int ROLE_WARPS = 4;      // warpgroup 0: weight producer, MMA issuer, stage watcher, activation producer
+constexpr int THREADS = 32 * (ROLE_WARPS + EPI_WARPS);
+constexpr int ROLE_REGS = 56, EPI_REGS = 224;   // registers per thread after the split: 128 * 56 + 256 * 224 <= 64 K
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int SMEM_BUDGET = 220 * 1024;
 constexpr int TMEM_COLS = 512;
@@ -117,6 +119,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t tmem_acc = tmem_base_slot;
   volatile int *abortp = &abort_flag;
 
+  // The epilogue warps hold the whole accumulator (144 registers per thread) next to their
+  // own arithmetic; at the kernel-wide limit of 168 the compiler serialises that arithmetic to
+  // save registers (SwiGLU: 1000 instead of 300 cycles per chunk) and spills in the argmax.  The
+  // four role warps need few registers, so their warpgroup hands most of its share over.
+  // (Each reallocation heads the code that runs under it, which is how the compiler learns
+  // the register budget of that code.)
+
+  if (warp < ROLE_WARPS) {
+  sm100::setmaxnreg_dec<ROLE_REGS>();
   if (warp == 0) {
     // ===================== weight producer =====================
     if (lane == 0) {
@@ -136,7 +147,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
       }
     }
-  } else if (warp == 3 + EPI_WARPS) {
+  } else if (warp == 3) {
     // ===================== activation producer =====================
     if (lane == 0) {
       sm100::prefetch_tensormap(&tmA);
@@ -212,7 +223,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       if (lane == 0) sm100::mma_commit(sm100::smem_u32(&tmem_full_bar));
       __syncwarp();
     }
-  } else if (warp == 2 + EPI_WARPS) {
+  } else if (warp == 2) {
     // ===================== stage watcher =====================
     // Waits (bounded) for the accumulator to be drained and for each stage's loads to land,
     // then arrives on the stage's hardware barrier.  A stage's barrier cannot be arrived on
@@ -239,11 +250,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (++sa == g.a_stages) { sa = 0; pha ^= 1u; }
       }
     }
-  } else if (warp >= 2 && warp < 2 + EPI_WARPS) {
+  }
+  } else {
+    sm100::setmaxnreg_inc<EPI_REGS>();
     // ===================== epilogue =====================
     pdl_wait();
     const int q = warp & 3;                      // TMEM lane quadrant this warp may read
-    const int half = (warp - 2) >> 2;
+    const int half = (warp - ROLE_WARPS) >> 2;
     const int hc = ((g.rb_rows / 2 + 15) / 16) * 16;
     const int c_begin = half ? hc : 0;
     const int c_end = half ? g.rb_rows : (hc < g.rb_rows ? hc : g.rb_rows);
@@ -329,7 +342,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         // through shared memory so that every lane stores 8 consecutive features of one
         // row with one 16-byte store: 2-byte stores from each lane took 18 us per tile.
         const bool odd = lane & 1;
-        uint16_t (*stage)[16] = epi_stage[warp - 2];
+        uint16_t (*stage)[16] = epi_stage[warp - ROLE_WARPS];
         const int srow = lane >> 1, sf = (lane & 1) * 8;
         const int f0 = ((tile * TILE_N + q * 32) >> 1) + sf;          // first of this lane's 8 features
         const int n_feat = g.N >> 1;

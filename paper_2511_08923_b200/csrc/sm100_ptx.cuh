@@ -58,6 +58,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// Register reallocation between warpgroups (all four warps of an aligned warpgroup execute
+// the same one).  dec releases registers to the SM's pool, inc waits until the pool has them.
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // ---- named barriers (hardware barriers 1..15 of the CTA; 0 is __syncthreads) -------------
 // Both are executed by whole, converged warps; `threads` counts every participating thread
 // (arriving and waiting) and is a multiple of 32.  Unlike an mbarrier test, waiting here does
