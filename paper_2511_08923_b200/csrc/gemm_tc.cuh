@@ -10,16 +10,16 @@
 // dimension) and the activation rows on the MMA N dimension (up to 288 = two instructions
 // of up to 144 columns), so no tensor-core work is wasted on padding rows.
 //
-// Work item = (row block, 128-row weight tile, K split).  Persistent CTAs, one per SM,
-// loop over items.  Warp roles: warp 0 streams weight tiles and warp 3 activation tiles by
-// TMA into two rings of shared-memory stages (the weight ring is the deep one: a tile comes
-// from HBM, takes > 1 us to arrive and is what bounds the kernel, while the wide activation
-// tile comes from L2 and only needs to be a little ahead), warp 1 issues the MMAs into one
-// fp32 accumulator in TMEM, warps 4..11 drain the
-// accumulator into registers (which frees it for the next item at once) and then run the
-// epilogue from registers while the next item's MMAs proceed, and warp 2 watches the
-// stages' mbarriers on behalf of the MMA warp (which must not touch the memory pipeline
-// between its MMAs) and releases it through hardware barriers.
+// Work item = (row block, 128-row weight tile, K split).  Persistent CTAs, one per SM, loop
+// over items.  Warp roles:
+//   warp 0      streams the weight tiles by TMA into a deep ring of shared-memory stages (a
+//               tile comes from HBM and takes > 1 us to arrive);
+//   warp 3      streams the wide activation tiles (from L2) into a ring of three stages;
+//   warp 1      issues the MMAs into one fp32 accumulator in TMEM;
+//   warp 2      watches the stages' mbarriers on behalf of warp 1, which must not touch the
+//               memory pipeline between its MMAs, and releases it through hardware barriers;
+//   warps 4-11  drain the accumulator into registers (which frees it for the next item at
+//               once) and run the epilogue from registers while the next item's MMAs proceed.
 #pragma once
 #include "common.cuh"
 #include "sm100_ptx.cuh"
