@@ -248,6 +248,23 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   if (mode == gemm_tc::MODE_SLAB) {
     a.n_tiles_b = a.n_tiles;
     a.S = force_S > 0 ? std::min(force_S, a.kb_total) : gemm_tc::plan_splits(a.n_rb * a.n_tiles, a.kb_total, c->n_sms, c->S_max, 4);
+    // One row block of up to 288 rows, or two of half the rows?  Two halves fetch every weight tile
+    // twice (the second time from L2: ~0.37 instead of 0.46 us per K block of an item, but twice as
+    // many K blocks per item once the SMs are full), while a CTA's slab store, which its SM cannot
+    // push out faster than ~42 GB/s, shrinks from 3.3 to 1.7 us and fewer slabs are left for the
+    // consumer.  Halves win when an item has few K blocks (the 1.5B-class shapes: step -6.5 %), one
+    // block when it has many (the 8B-class shapes: halves cost +4 %).
+    if (force_S <= 0 && a.n_rb == 1 && R > gemm_tc::MAX_ROWS / 2) {
+      gemm_tc::Args h = a;
+      gemm_tc::plan_rows(R, h, gemm_tc::MAX_ROWS / 2);
+      h.S = gemm_tc::plan_splits(h.n_rb * h.n_tiles, h.kb_total, c->n_sms, c->S_max, 4);
+      auto cost = [&](const gemm_tc::Args &x, double us_per_kb, double us_store) {
+        const long long items = (long long)x.n_rb * x.n_tiles * x.S;
+        const long long waves = (items + c->n_sms - 1) / c->n_sms;
+        return waves * ((x.kb_total + x.S - 1) / x.S * us_per_kb + 1.5) + us_store + 0.5 * x.S;
+      };
+      if (cost(h, 0.37, 1.7) < cost(a, 0.46, 3.3)) a = h;
+    }
     a.out = slab_out ? (void *)slab_out : (void *)c->partials; a.ldo = N; a.slab_stride = (long long)R * N;
     a.slab_bf16 = (slab_out || !c->slab_bf16) ? 0 : 1;   // an explicit output buffer always gets exact fp32 slabs
   } else if (mode == gemm_tc::MODE_SWIGLU) {
