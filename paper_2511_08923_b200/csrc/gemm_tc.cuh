@@ -34,7 +34,7 @@ constexpr int ROLE_WARPS = 4;      // warpgroup 0: weight producer, MMA issuer, 
 constexpr int THREADS = 32 * (ROLE_WARPS + EPI_WARPS);
 constexpr int ROLE_REGS = 56, EPI_REGS = 224;   // registers per thread after the split: 128 * 56 + 256 * 224 <= 64 K
 constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
-constexpr int SMEM_BUDGET = 220 * 1024;
+constexpr int SMEM_BUDGET = 216 * 1024;   // dynamic shared memory for the rings; up to 9 KB of static shared memory come on top
 constexpr int TMEM_COLS = 512;
 
 enum Mode { MODE_SLAB = 0, MODE_SWIGLU = 1, MODE_ARGMAX = 2 };
@@ -89,7 +89,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ __align__(8) uint64_t w_full[8], w_empty[8], a_full[8], a_empty[8], tmem_full_bar, tmem_empty_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ __align__(16) uint16_t epi_stage[MODE == MODE_SWIGLU ? EPI_WARPS : 1][16][16];   // MODE_SWIGLU: one 16-column chunk per epilogue warp, [column][feature]
+  __shared__ __align__(16) uint16_t epi_stage[MODE == MODE_SWIGLU ? EPI_WARPS : 1][32][16];   // MODE_SWIGLU: two 16-column chunks per epilogue warp, [column][feature]
 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -346,36 +346,52 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int srow = lane >> 1, sf = (lane & 1) * 8;
         const int f0 = ((tile * TILE_N + q * 32) >> 1) + sf;          // first of this lane's 8 features
         const int n_feat = g.N >> 1;
+        // Two 16-column chunks per pass: all exchanges first, then sixteen independent silu
+        // chains (one chain at a time is bound by instruction latency: 16 us per tile instead of
+        // 2), then the turn through shared memory.
 #pragma unroll
-        for (int i = 0; i < 9; ++i) {
-          if (i * 16 < ncols) {
-            // exchanges first, then eight independent silu chains: one chain at a time is
-            // bound by instruction latency (16 us per tile instead of 2)
-            uint32_t recv[8];
+        for (int ip = 0; ip < 5; ++ip) {
+          if (ip * 32 < ncols) {
+            const bool second = (2 * ip + 1) < 9 && (2 * ip + 1) * 16 < ncols;      // warp-uniform
+            float h[2][8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) recv[j] = __shfl_xor_sync(0xffffffffu, odd ? v[i][2 * j] : v[i][2 * j + 1], 1);
-            float h[8];
+            for (int c = 0; c < 2; ++c) {
+              const int i = (2 * ip + c) < 9 ? 2 * ip + c : 8;
+              if (c == 0 || second) {
+                uint32_t recv[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float gate = __uint_as_float(odd ? recv[j] : v[i][2 * j]);
-              const float up = __uint_as_float(odd ? v[i][2 * j + 1] : recv[j]);
-              h[j] = silu_mul(gate, up);
-            }
+                for (int j = 0; j < 8; ++j) recv[j] = __shfl_xor_sync(0xffffffffu, odd ? v[i][2 * j] : v[i][2 * j + 1], 1);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) stage[2 * j + (odd ? 1 : 0)][lane >> 1] = __bfloat16_as_ushort(__float2bfloat16(h[j]));
-            __syncwarp();
-            const uint4 packed = *reinterpret_cast<const uint4 *>(&stage[srow][sf]);
-            const int r = r_base + i * 16 + srow;
-            if (r < g.R) {
-              bf16 *dst = g.H + (long long)r * g.ldh + f0;
-              if (f0 + 8 <= n_feat && (g.ldh & 7) == 0) {
-                *reinterpret_cast<uint4 *>(dst) = packed;
-              } else {
-                const uint16_t *e = reinterpret_cast<const uint16_t *>(&packed);
-                for (int t = 0; t < 8; ++t)
-                  if (f0 + t < n_feat) dst[t] = __ushort_as_bfloat16(e[t]);
+                for (int j = 0; j < 8; ++j) {
+                  const float gate = __uint_as_float(odd ? recv[j] : v[i][2 * j]);
+                  const float up = __uint_as_float(odd ? v[i][2 * j + 1] : recv[j]);
+                  h[c][j] = silu_mul(gate, up);
+                }
               }
             }
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+              if (c == 0 || second) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) stage[c * 16 + 2 * j + (odd ? 1 : 0)][lane >> 1] = __bfloat16_as_ushort(__float2bfloat16(h[c][j]));
+              }
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+              if (c == 0 || second) {
+                const uint4 packed = *reinterpret_cast<const uint4 *>(&stage[c * 16 + srow][sf]);
+                const int r = r_base + (2 * ip + c) * 16 + srow;
+                if (r < g.R) {
+                  bf16 *dst = g.H + (long long)r * g.ldh + f0;
+                  if (f0 + 8 <= n_feat && (g.ldh & 7) == 0) {
+                    *reinterpret_cast<uint4 *>(dst) = packed;
+                  } else {
+                    const uint16_t *e = reinterpret_cast<const uint16_t *>(&packed);
+                    for (int t = 0; t < 8; ++t)
+                      if (f0 + t < n_feat) dst[t] = __ushort_as_bfloat16(e[t]);
+                  }
+                }
+              }
             __syncwarp();
           }
         }

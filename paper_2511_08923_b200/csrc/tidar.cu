@@ -353,12 +353,17 @@ bool encode_local_map(tidar_ctx *c, CUtensorMap *tm, const void *loc, long long 
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Key-range split of the attention kernel: fill the SMs (two CTAs fit on one) without
-// giving a CTA fewer than two key tiles.
+// Key-range split of the attention kernel: fill the SMs (two CTAs fit on one) without giving a
+// CTA fewer than two key tiles; and once half the SMs have a CTA, not fewer than five: a CTA pays
+// ~7 us of set-up, partial-result store and merge traffic whatever its key range (1.5B-class
+// step at n = 1 k: 8 splits 585 us per 4 layers, 4 splits 571), while a nearly empty machine
+// (the k = 1 step) is served best by as many CTAs as there are key tiles to hand out.
 int attn_key_splits(const tidar_ctx *c, int units, int key_tiles_hint) {
   int splits = 2 * c->n_sms / std::max(units, 1);
   splits = std::min(splits, std::max(1, key_tiles_hint / 2));
-  return std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
+  splits = std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
+  while (splits > 1 && units * splits > c->n_sms / 2 && key_tiles_hint / splits < 5) --splits;
+  return splits;
 }
 
 struct AttnMaps { const CUtensorMap *q, *k, *v, *kloc, *vloc; int page_base_k, page_base_v; };
