@@ -181,18 +181,34 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   *bytes = align_up(cv.off, 256);
 }
 
-// Launch with programmatic stream serialization: the kernel may be scheduled while the
-// previous kernel of the stream is still running and synchronises itself with pdl_wait().
-// Only kernels that call pdl_wait() before touching produced data may be launched this way.
+// Two ways to launch a kernel of the step.  launch_pdl: with programmatic stream serialization,
+// the kernel may be scheduled while the previous kernel of the stream is still running and
+// synchronises itself with pdl_wait(); only kernels that call pdl_wait() before touching
+// produced data may be launched this way.  It pays for kernels with a heavy prologue (the
+// projections: tensor-memory allocation, barriers, the weight ring filling; attention).
+// launch_after: an ordinary dependency.  The small kernels gain nothing from starting early,
+// and their CTAs waiting on the SMs only take resources from the kernel that is still
+// running: a chain of small kernels in a graph costs ~1 us per kernel either way (1.5B-class
+// step 2.57 -> 2.51 ms, k = 1 step 1.71 -> 1.59 ms with the small kernels launched this way).
+// Their pdl_wait() / pdl_trigger() are no-ops then, apart from letting the NEXT kernel start
+// early.
 template <typename... KP, typename... AP>
-inline void launch_pdl(void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AP &&...args) {
+inline void launch_with(bool programmatic, void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AP &&...args) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
+  cfg.attrs = at; cfg.numAttrs = programmatic ? 1 : 0;
   cudaLaunchKernelEx(&cfg, kernel, KP(std::forward<AP>(args))...);
+}
+template <typename... KP, typename... AP>
+inline void launch_pdl(void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AP &&...args) {
+  launch_with(true, kernel, grid, block, smem, st, std::forward<AP>(args)...);
+}
+template <typename... KP, typename... AP>
+inline void launch_after(void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AP &&...args) {
+  launch_with(false, kernel, grid, block, smem, st, std::forward<AP>(args)...);
 }
 
 // ---- launch bookkeeping -----------------------------------------------------
@@ -302,10 +318,10 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     const size_t n = (size_t)R * nf;
     c->launches++;
     if (c->slab_bf16)
-      launch_pdl(swiglu_slab_kernel<bf16>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+      launch_after(swiglu_slab_kernel<bf16>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
                                                                            a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
     else
-      launch_pdl(swiglu_slab_kernel<float>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const float *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
+      launch_after(swiglu_slab_kernel<float>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const float *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
                                                                            a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
   }
   if (S_out) *S_out = a.S;
@@ -397,9 +413,9 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
     Launch l(c, TIDAR_TC_ATTN);
     const int warps = R * cf.n_q_heads;
     if (cf.head_dim == 128)
-      launch_pdl(attn_tc::attn_combine_kernel<128>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<128>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
     else
-      launch_pdl(attn_tc::attn_combine_kernel<64>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<64>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
   }
 }
 
@@ -419,9 +435,9 @@ void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t strid
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
   if (c->cfg.impl == 0 && c->slab_bf16)
-    launch_pdl(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+    launch_after(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
   else
-    launch_pdl(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+    launch_after(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
 }
 
 // The transformer stack over R assembled rows (metadata and X already filled).
@@ -433,7 +449,7 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
   {
     Launch l(c, TIDAR_TC_ROPE);
     const int n = R * (hd / 2);
-    launch_pdl(rope_table_kernel, (n + 255) / 256, 256, 0, c->stream, c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
+    launch_after(rope_table_kernel, (n + 255) / 256, 256, 0, c->stream, c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
   }
   int S = 0; size_t stride = 0;          // pending partials of the previous down projection
   const bool tc = cf.impl == 0;
@@ -450,10 +466,10 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
       Launch ll(c, TIDAR_TC_ROPE);
       const int rope_chunks = ((Hq + 2 * Hkv) * (hd / 8) + 255) / 256;
 if (tc && c->slab_bf16)
-        launch_pdl(rope_kv_kernel<bf16>, dim3(R, rope_chunks), 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+        launch_after(rope_kv_kernel<bf16>, dim3(R, rope_chunks), 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
       else
-        launch_pdl(rope_kv_kernel<float>, dim3(R, rope_chunks), 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
+        launch_after(rope_kv_kernel<float>, dim3(R, rope_chunks), 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
                                                                       c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
     }
     if (tc) {
@@ -483,7 +499,7 @@ if (tc && c->slab_bf16)
     CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
     if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    launch_pdl(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
+    launch_after(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
@@ -581,18 +597,18 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint) {
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
-    launch_pdl(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
+    launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
                c->d_step_n, c->embed, cf.d_model, c->X);
   }
   if (int rc = forward_rows(c, R, true, T, key_tiles_hint)) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    launch_pdl(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
+    launch_after(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
                c->d_step_L, c->d_out);
   }
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    launch_pdl(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
+    launch_after(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
                (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
   }
   CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
