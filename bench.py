@@ -47,8 +47,8 @@ def peaks():
 # ----------------------------------------------------------------------------
 # algorithmic cost of one step (per sequence)
 # ----------------------------------------------------------------------------
-def step_cost(sh, k, n, n_layers=None):
-    """Algorithmic bytes and flops of one decode step with n cached positions.
+def step_cost(sh, k, n, n_layers=None, batch=1):
+    """Algorithmic bytes and flops of one decode step of `batch` sequences with n cached positions each.
 
     bytes: every projection weight and the LM head once (bf16) + the K/V of the n
     cached positions once per layer.  flops: 2*T*params for the projections +
@@ -63,6 +63,7 @@ def step_cost(sh, k, n, n_layers=None):
     # keys per row: causal j sees n+j+1, mask (b, .) sees n+b+1+k
     keys = sum(n + j + 1 for j in range(k)) + sum(k * (n + b + 1 + k) for b in range(k))
     attn_flops = L * 4 * sh.n_q_heads * sh.head_dim * keys
+    kv_bytes *= batch; attn_flops *= batch; T *= batch      # weights are shared, everything else is per sequence
     return {"T": T, "params": params, "weight_bytes": 2 * params, "kv_bytes": kv_bytes,
             "gemm_flops": 2 * T * params, "attn_flops": attn_flops,
             "bytes": 2 * params + kv_bytes, "flops": 2 * T * params + attn_flops}
@@ -227,6 +228,8 @@ def main():
     ap.add_argument("--kernels", type=int, default=None, help="library impl: 0 tensor-core, 1 replay (diagnostic)")
     ap.add_argument("--layers", type=int, default=None, help="reduced-depth twin (diagnostics only; not a bench value)")
     ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=1, help="sequences decoded together (the batch / block sweep; default 1)")
+    ap.add_argument("--prompt-len", type=int, default=None, help="cached positions per sequence at the start (default: the workload's)")
     ap.add_argument("--per-l-steps", type=int, default=2)
     ap.add_argument("--ar-steps", type=int, default=32, help="steps of the k = 1 autoregressive reference (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -239,7 +242,8 @@ def main():
     if args.layers:
         sh = sh.reduced(args.layers)
     k = args.k or sh.k
-    n0 = sh.prompt_len
+    n0 = args.prompt_len or sh.prompt_len
+    B = args.batch
     if args.impl == "reference":
         run_reference(args, sh, k, n0)
         return
@@ -263,11 +267,16 @@ def main():
     torch.cuda.empty_cache()
     stream = torch.cuda.Stream(device=dev)
     n_steps_total = args.warmup + 2 * args.steps + 8 + k * args.per_l_steps
-    t = Tidar(sh, packed, k_max=k, max_batch=1, max_seq_len=n0 + (n_steps_total + 4) * k + 2 * k + 64, impl=impl,
+    t = Tidar(sh, packed, k_max=k, max_batch=B, max_seq_len=n0 + (n_steps_total + 4) * k + 2 * k + 64, impl=impl,
               device=dev, stream=stream, debug=args.lib_debug)
     prompt = gen_token_ids(sh.seed, tensor_id("prompt"), n0, sh.vocab - 1).numpy()
-    t.prefill(0, prompt, k)
-    sched = acceptance_schedule(SCHEDULE_SEED, args.warmup + 2 * args.steps, k).numpy()
+    seqs = list(range(B))
+    for b in seqs:
+        t.prefill(b, np.roll(prompt, b), k)
+    sched = acceptance_schedule(SCHEDULE_SEED, args.warmup + 2 * args.steps + B, k).numpy()
+
+    def forced(si, L=None):           # sequence b of step si takes the schedule's entry si + b
+        return [int(sched[si + b]) if L is None else L for b in seqs]
 
     def barrier():
         if world > 1:
@@ -277,7 +286,7 @@ def main():
     # ---- device-resident timing: K steps, CUDA events on the library's stream -----
     si = 0
     for _ in range(args.warmup):
-        t.step_async([0], [int(sched[si])]); t.step_wait(); si += 1
+        t.step_async(seqs, forced(si)); t.step_wait(); si += 1
     n_start = t.seq_len(0)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = t.launch_count()
@@ -287,7 +296,7 @@ def main():
             ev0.record(stream)
         tokens = 0
         for _ in range(args.steps):
-            t.step_async([0], [int(sched[si])]); _, L = t.step_wait(); tokens += L[0]; si += 1
+            t.step_async(seqs, forced(si)); _, L = t.step_wait(); tokens += sum(L); si += 1
         with torch.cuda.stream(stream):
             ev1.record(stream)
         barrier()
@@ -301,7 +310,7 @@ def main():
     w0 = time.perf_counter()
     tokens_e2e = 0
     for _ in range(args.steps):
-        _, L = t.step([0], [int(sched[si])]); tokens_e2e += L[0]; si += 1
+        _, L = t.step(seqs, forced(si)); tokens_e2e += sum(L); si += 1
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
 
@@ -310,30 +319,30 @@ def main():
     cls = {}
     n_t = 4
     for _ in range(n_t):
-        t.step([0], [8 if k >= 8 else k])
+        t.step(seqs, forced(0, 8 if k >= 8 else k))
         for kk, v in t.timing().items():
             cls[kk] = cls.get(kk, 0.0) + v / n_t
     t.set_timing(False)
 
     # ---- per acceptance length -----------------------------------------------------------
     per_L = {}
-    for L in range(1, k + 1):
+    for L in (range(1, k + 1) if args.per_l_steps > 0 else ()):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record(stream)
         for _ in range(args.per_l_steps):
-            t.step_async([0], [L]); t.step_wait()
+            t.step_async(seqs, forced(0, L)); t.step_wait()
         b.record(stream)
         torch.cuda.synchronize()
         ms = a.elapsed_time(b) / args.per_l_steps
-        per_L[str(L)] = {"ms_per_step": round(ms, 4), "tokens_per_s": round(L / ms * 1e3, 1)}
+        per_L[str(L)] = {"ms_per_step": round(ms, 4), "tokens_per_s": round(B * L / ms * 1e3, 1)}
 
     # ---- autoregressive reference on the same kernels: k = 1 (one settled token per pass) ----
     # The paper's headline is decode tokens/s relative to plain AR decoding of the same model
     # (Section 4.3); this gives the same ratio on this GPU.  A k = 1 step carries one causal slot
     # and one mask slot and always emits exactly one token.
     ar = None
-    if args.ar_steps > 0:
+    if args.ar_steps > 0 and B == 1:
         t.close()
         t = Tidar(sh, packed, k_max=1, max_batch=1, max_seq_len=n0 + args.ar_steps + 16, impl=impl, device=dev, stream=stream,
                   debug=args.lib_debug)
@@ -357,7 +366,7 @@ def main():
     if rank == 0:
         pk, pk_src = peaks()
         ms_step = ms_total / args.steps
-        cost = step_cost(sh, k, n_mid)
+        cost = step_cost(sh, k, n_mid, batch=B)
         t_hbm = cost["bytes"] / (pk["hbm_gbs"] * 1e9) * 1e3
         t_tensor = cost["flops"] / (pk["bf16_tflops_sustained"] * 1e12) * 1e3
         t_hbm_nom = cost["bytes"] / (NOMINAL["hbm_gbs"] * 1e9) * 1e3
@@ -375,7 +384,7 @@ def main():
         else:
             ach = cost["weight_bytes"] / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
             roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s"}
-        tr = TRAFFIC.get(args.workload)
+        tr = TRAFFIC.get(args.workload) if (B == 1 and k == sh.k and not args.layers and not args.prompt_len) else None
         roof.update({"frac": roof["achieved"] / roof["peak"],
                      "traffic": tr["bytes_per_step"] if tr else None,
                      "traffic_note": tr["note"] if tr else "no ncu capture of this workload since the kernel last changed",
@@ -386,15 +395,15 @@ def main():
         line = {"metric": "decode_tokens_per_s", "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": workload_config(sh, k, n0, 1), "clocks": clocks,
-                "e2e": {"value": tokens_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": 8, "d2h_bytes_per_step": 4 * (k + 1),
+                "config": workload_config(sh, k, n0, B), "clocks": clocks,
+                "e2e": {"value": tokens_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": 8 * B, "d2h_bytes_per_step": 4 * (k + 1) * B,
                         "ms_per_step": 1e3 * e2e_s / args.steps},
                 "gpu_launches": int(launches),
                 "roofline": roof,
                 "step_roofline": {"bytes": cost["bytes"], "flops": cost["flops"], "n_cached": n_mid,
                                   "t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor, "frac_measured_peaks": max(t_hbm, t_tensor) / ms_step,
                                   "frac_nominal_peaks": max(t_hbm_nom, t_tensor_nom) / ms_step, "peaks": pk, "peak_source": pk_src},
-                "mean_accept_len": tokens / (args.steps * world), "per_accept_len": per_L,
+                "mean_accept_len": tokens / (args.steps * world * B), "per_accept_len": per_L,
                 "ar_reference": ar,
                 "kernels": "tcgen05" if impl == 0 else "replay (fp32 CUDA cores)",
                 "paper_context": "paper reports 4.71x (1.5B) / 5.91x (8B) tokens/s over AR on one H100; no absolute figure"}
