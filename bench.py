@@ -209,6 +209,42 @@ def run_reference(args, sh, k, n0):
     print(json.dumps(line))
 
 
+def attention_microbench(reps=50):
+    """Structured-mask attention alone (`tidar_attention`: row table, attention kernel, merge of the key
+    splits) at 32/8 heads, head_dim 128, k = 16 and 1 k .. 32 k cached positions in shuffled pages; one
+    JSON line per length.  A diagnostic beside the step benchmark, not a bench value."""
+    from dataclasses import replace
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    hd, Hq, Hkv, k = 128, 32, 8, 16
+    sh = replace(CONFIGS["tiny"], head_dim=hd, n_q_heads=Hq, n_kv_heads=Hkv, n_layers=1, vocab=64, d_ffn=64, d_model=64)
+    t = Tidar(sh, pack_weights(gen_model_weights(sh), "cuda:0"), k_max=k, max_batch=1, max_seq_len=128, impl=0)
+    T = k * (k + 1)
+    pk, _ = peaks()
+    g = torch.Generator(device="cuda:0"); g.manual_seed(7)
+    rnd = lambda *shape: torch.randn(*shape, device="cuda:0", generator=g).bfloat16()
+    for n in (1024, 4096, 16384, 32768):
+        pps = (n + k + 63) // 64
+        q, kp, vp, kl, vl = rnd(T, Hq, hd), rnd(pps, Hkv, 64, hd), rnd(pps, Hkv, 64, hd), rnd(k * k, Hkv, hd), rnd(k * k, Hkv, hd)
+        pt = torch.randperm(pps, device="cuda:0", generator=g).to(torch.int32).view(1, pps)
+        sl = torch.tensor([n], dtype=torch.int32, device="cuda:0")
+        out = torch.empty(T, Hq * hd, dtype=torch.bfloat16, device="cuda:0")
+        for _ in range(3):
+            t.attention(q, kp, vp, pt, sl, kl, vl, out, 1, k)
+        t.sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            t.attention(q, kp, vp, pt, sl, kl, vl, out, 1, k)
+        e1.record(); torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        keys = sum(n + j + 1 for j in range(k)) + sum(k * (n + b + 1 + k) for b in range(k))
+        flops, nbytes = 4 * Hq * hd * keys, n * Hkv * hd * 2 * 2
+        print(json.dumps({"attention_microbench": {"cached_positions": n, "k": k, "heads": f"{Hq}/{Hkv}", "head_dim": hd},
+                          "us_per_call": round(us, 1), "tflops": round(flops / us / 1e6, 1), "kv_gbs": round(nbytes / us / 1e3, 1),
+                          "frac_of_measured_bf16_peak": round(flops / us / 1e6 / pk["bf16_tflops_sustained"], 3)}))
+    t.close()
+
+
 def workload_config(sh, k, n0, batch):
     return {"workload": f"TiDAR decode step, {sh.name}-class decoder ({sh.n_layers} layers, d_model {sh.d_model}, "
                         f"{sh.n_q_heads}/{sh.n_kv_heads} heads, head_dim {sh.head_dim}, ffn {sh.d_ffn}, vocab {sh.vocab}), "
@@ -233,6 +269,7 @@ def main():
     ap.add_argument("--per-l-steps", type=int, default=2)
     ap.add_argument("--ar-steps", type=int, default=32, help="steps of the k = 1 autoregressive reference (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--attn-microbench", action="store_true", help="time the attention entry point alone at 1 k .. 32 k cached positions and exit")
     ap.add_argument("--lib-debug", type=int, default=0, help="library debug bits (4: bf16 split-K partial sums; diagnostics, not the bench configuration)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -248,6 +285,11 @@ def main():
         run_reference(args, sh, k, n0)
         return
 
+    if args.attn_microbench:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        attention_microbench()
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
     rank = int(os.environ.get("RANK", "0"))
