@@ -368,7 +368,12 @@ def main():
 
     # ---- per acceptance length -----------------------------------------------------------
     per_L = {}
+    # every L starts from the same context (a fresh first pass over the prompt and one untimed
+    # step), so that the latencies differ by L alone and not by how far the cache has grown
     for L in (range(1, k + 1) if args.per_l_steps > 0 else ()):
+        for b_ in seqs:
+            t.prefill(b_, np.roll(prompt, b_), k)
+        t.step_async(seqs, forced(0, L)); t.step_wait()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record(stream)
