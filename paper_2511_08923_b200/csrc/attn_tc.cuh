@@ -385,30 +385,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 }
 
 // Merge the per-split partial results: O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
-// One warp per (row, head).
+// HD / 4 threads per (row, head), four consecutive columns each: 16-byte loads, 8-byte stores.
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
                                bf16 *__restrict__ O) {
   pdl_trigger();
   pdl_wait();
-  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (wid >= R * Hq) return;
+  constexpr int PER = HD / 4;
+  const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t wid = gid / PER;
+  const int c4 = (int)(gid % PER);
+  if (wid >= (size_t)R * Hq) return;
   float M = -INFINITY;
   for (int s = 0; s < splits; ++s) M = fmaxf(M, part_ml[((size_t)s * R * Hq + wid) * 2]);
-  float den = 0.f, acc[HD / 32];
-#pragma unroll
-  for (int i = 0; i < HD / 32; ++i) acc[i] = 0.f;
+  float den = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int s = 0; s < splits; ++s) {
     const size_t idx = (size_t)s * R * Hq + wid;
     const float m = part_ml[idx * 2], l = part_ml[idx * 2 + 1];
     const float wgt = (m == -INFINITY) ? 0.f : exp2f(m - M);
     den += wgt * l;
-#pragma unroll
-    for (int i = 0; i < HD / 32; ++i) acc[i] = fmaf(wgt, part_O[idx * HD + i * 32 + lane], acc[i]);
+    const float4 v = reinterpret_cast<const float4 *>(part_O + idx * HD)[c4];
+    acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y); acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
   }
   const float inv = 1.f / den;
-#pragma unroll
-  for (int i = 0; i < HD / 32; ++i) O[(size_t)wid * HD + i * 32 + lane] = __float2bfloat16(acc[i] * inv);
+  __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  uint2 u; u.x = *reinterpret_cast<uint32_t *>(&h0); u.y = *reinterpret_cast<uint32_t *>(&h1);
+  reinterpret_cast<uint2 *>(O + wid * HD)[c4] = u;
 }
 
 }  // namespace attn_tc

@@ -411,11 +411,11 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   }
   if (a.splits > 1) {
     Launch l(c, TIDAR_TC_ATTN);
-    const int warps = R * cf.n_q_heads;
+    const size_t threads = (size_t)R * cf.n_q_heads * (cf.head_dim / 4);
     if (cf.head_dim == 128)
-      launch_after(attn_tc::attn_combine_kernel<128>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<128>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
     else
-      launch_after(attn_tc::attn_combine_kernel<64>, (warps + 7) / 8, 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<64>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
   }
 }
 
