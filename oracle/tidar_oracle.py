@@ -68,6 +68,11 @@ class OracleConfig:
     rms_eps: float
     mask_token_id: int
     beta: float = 1.0
+    # "f64": nothing is rounded (the definition).  "bf16": the activations a bf16 decoder keeps between
+    # its operators (normed inputs of the projections, Q, K, V after RoPE, the attention output, the
+    # SwiGLU output) are rounded to bfloat16 where they are stored; the paper trains and runs in
+    # "standard BFloat 16" (Section 4.1).  All arithmetic stays float64 in both modes.
+    act_dtype: str = "f64"
 
 
 @dataclass
@@ -171,6 +176,24 @@ def build_prefill_mask(n: int, k: int) -> np.ndarray:
 # ----------------------------------------------------------------------------
 # layers
 # ----------------------------------------------------------------------------
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 (ties to even) of every element, returned as float64.
+
+    bfloat16 is the upper half of an IEEE float32: the value is first taken to float32, then the low
+    16 bits are rounded away (add 0x7FFF plus the lowest kept bit, clear the low half)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(F64)
+
+
+def _stored(cfg: "OracleConfig", x: np.ndarray) -> np.ndarray:
+    """An activation as the next operator reads it: unchanged, or rounded to bf16 (cfg.act_dtype)."""
+    if cfg.act_dtype == "f64":
+        return x
+    assert cfg.act_dtype == "bf16", cfg.act_dtype
+    return round_bf16(x)
+
+
 def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
     ms = np.mean(x * x, axis=-1, keepdims=True)
     return x / np.sqrt(ms + eps) * gain
@@ -226,21 +249,21 @@ def forward(cfg: OracleConfig, w: dict, ids: np.ndarray, pos: np.ndarray, mask: 
     hidden, k_new, v_new = [], [], []
     for l, L in enumerate(w["layers"]):
         hidden.append(x.copy())
-        a = rmsnorm(x, L["attn_norm"], cfg.rms_eps)
+        a = _stored(cfg, rmsnorm(x, L["attn_norm"], cfg.rms_eps))
         q = (a @ L["wq"].T).reshape(R, Hq, hd)
         kk = (a @ L["wk"].T).reshape(R, Hkv, hd)
-        vv = (a @ L["wv"].T).reshape(R, Hkv, hd)
-        q = rope(q, pos, cfg.rope_theta)
-        kk = rope(kk, pos, cfg.rope_theta)
+        vv = _stored(cfg, (a @ L["wv"].T).reshape(R, Hkv, hd))
+        q = _stored(cfg, rope(q, pos, cfg.rope_theta))
+        kk = _stored(cfg, rope(kk, pos, cfg.rope_theta))
         k_new.append(kk); v_new.append(vv)
         k_all = np.concatenate([k_cache[l], kk], axis=0) if len(k_cache[l]) else kk
         v_all = np.concatenate([v_cache[l], vv], axis=0) if len(v_cache[l]) else vv
-        o = masked_attention(q, k_all, v_all, mask).reshape(R, Hq * hd)
+        o = _stored(cfg, masked_attention(q, k_all, v_all, mask).reshape(R, Hq * hd))
         x = x + o @ L["wo"].T
-        f = rmsnorm(x, L["ffn_norm"], cfg.rms_eps)
-        x = x + swiglu(f @ L["w_gate"].T, f @ L["w_up"].T) @ L["w_down"].T
+        f = _stored(cfg, rmsnorm(x, L["ffn_norm"], cfg.rms_eps))
+        x = x + _stored(cfg, swiglu(f @ L["w_gate"].T, f @ L["w_up"].T)) @ L["w_down"].T
     hidden.append(x.copy())
-    y = rmsnorm(x, w["final_norm"], cfg.rms_eps)
+    y = _stored(cfg, rmsnorm(x, w["final_norm"], cfg.rms_eps))
     if logit_rows is None:
         logits = y @ w["lm_head"].T
     else:

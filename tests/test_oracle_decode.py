@@ -155,15 +155,63 @@ def test_first_mask_slot_and_ar_row_predict_the_same_position(model):
         assert pos[sh.k + b * sh.k] == pos[b] + 1
 
 
-def test_beta_mixes_logits_for_verification(model):
+def test_beta_endpoints_select_one_head_each(model):
+    """Section 4.4.3 pinned without the oracle's own mixing formula: at beta = 1 the verified targets are
+    the argmax of the causal rows alone, at beta = 0 the argmax of the first slot of each block alone
+    (each compared with the logits of an UNMIXED run), and the settled first token of the prefill
+    switches between the last prompt row and the first mask row in the same way."""
     sh, cfg, w, prompt = model
-    for beta in (1.0, 0.5, 0.0):
+    n, k = len(prompt), sh.k
+    runs = {}
+    for beta in (1.0, 0.0):
         cfg_b = replace(cfg, beta=beta)
-        st, _ = O.prefill(cfg_b, w, prompt, sh.k)
+        st, c, fo = O.prefill(cfg_b, w, prompt, k, return_forward=True)
+        st.block = np.array(runs[1.0][0] if beta == 0.0 else st.block)      # same drafts in both runs
+        block = st.block.copy()
         so = O.step(cfg_b, w, st)
-        a = so.fwd.logits[:sh.k]
-        g0 = so.fwd.logits[sh.k:].reshape(sh.k, sh.k, -1)[:, 0]
-        np.testing.assert_array_equal(so.targets, np.argmax(beta * a + (1 - beta) * g0, axis=-1))
+        runs[beta] = (block, c, fo, so)
+    _, c1, fo1, so1 = runs[1.0]
+    _, c0, fo0, so0 = runs[0.0]
+    np.testing.assert_array_equal(fo1.logits, fo0.logits)                   # beta does not touch the forward pass
+    assert c1 == int(np.argmax(fo1.logits[n - 1])) and c0 == int(np.argmax(fo1.logits[n]))
+    a = so1.fwd.logits[:k]
+    g0 = so1.fwd.logits[k:].reshape(k, k, -1)[:, 0]
+    np.testing.assert_array_equal(so1.targets, a.argmax(-1))
+    # the beta = 0 run starts from a different settled token, so compare on its own unmixed logits
+    a_0 = so0.fwd.logits[:k]; g0_0 = so0.fwd.logits[k:].reshape(k, k, -1)[:, 0]
+    np.testing.assert_array_equal(so0.targets, g0_0.argmax(-1))
+    assert not np.array_equal(a_0.argmax(-1), g0_0.argmax(-1)) or not np.array_equal(a.argmax(-1), g0.argmax(-1)), \
+        "the two heads agree everywhere on this input: the endpoints are not told apart"
+
+
+def test_beta_mix_on_hand_built_logits():
+    """The mixing rule on three-logit rows worked by hand (not by the oracle's expression): the
+    autoregressive row prefers id 0, the diffusion row id 2."""
+    a = np.array([[2.0, 1.0, 0.0]]); g0 = np.array([[0.0, 1.0, 4.0]])
+    # beta = 0.5: [1.0, 1.0, 2.0] -> id 2;  beta = 0.75: [1.5, 1.0, 1.0] -> id 0;  beta = 2/3: [4/3, 1, 4/3] ties -> lowest id 0
+    hand = {1.0: 0, 0.0: 2, 0.5: 2, 0.75: 0}
+    for beta, want in hand.items():
+        mixed = np.array([[beta * 2.0 + (1 - beta) * 0.0, 1.0, (1 - beta) * 4.0]])
+        assert int(O.argmax_lowest(mixed)[0]) == want
+        assert int(O.argmax_lowest(beta * a + (1.0 - beta) * g0)[0]) == want
+    assert int(O.argmax_lowest(np.array([[1.25, 1.0, 1.25]]))[0]) == 0      # ties go to the lowest id
+
+
+def test_beta_half_step_uses_the_mixed_row(model):
+    """beta = 0.5 in a real step: the targets are neither head's argmax in general, and on every slot
+    they beat both heads' choices under the mixed score (checked through the scores, not the argmax)."""
+    sh, cfg, w, prompt = model
+    k = sh.k
+    cfg_b = replace(cfg, beta=0.5)
+    st, _ = O.prefill(cfg_b, w, prompt, k)
+    so = O.step(cfg_b, w, st)
+    a = so.fwd.logits[:k]
+    g0 = so.fwd.logits[k:].reshape(k, k, -1)[:, 0]
+    for j in range(k):
+        score = lambda v: 0.5 * a[j, v] + 0.5 * g0[j, v]
+        tj = int(so.targets[j])
+        assert score(tj) >= score(int(a[j].argmax())) and score(tj) >= score(int(g0[j].argmax()))
+        assert score(tj) >= max(score(v) for v in range(0, sh.vocab, 7))
 
 
 # ---------------------------------------------------------------- planted mistakes must be caught

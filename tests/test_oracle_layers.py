@@ -163,3 +163,38 @@ def test_causal_forward_matches_transformers_llama(tied):
     # the library builds its rotary tables in float32, so agreement stops near 1e-7;
     # any structural mistake (pairing, head mapping, norm placement) is >= 1e-2
     np.testing.assert_allclose(fo.logits, ref, rtol=0, atol=2e-6)
+
+
+# ---- optional bf16 storage of activations (OracleConfig.act_dtype) -------------------------------
+def test_round_bf16_is_round_to_nearest_even_bfloat16():
+    """Pinned against torch's float32 -> bfloat16 conversion and against hand-worked bit patterns."""
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096), [0.0, -0.0, 1.0, -1.0, 3.0e38, 1e-40]])
+    want = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(O.round_bf16(x), want)
+    # 1 + 2^-8 lies exactly between 1 and 1 + 2^-7: ties go to the even mantissa (1.0);
+    # 1 + 3 * 2^-8 lies between 1 + 2^-7 (odd) and 1 + 2^-6 (even): up
+    np.testing.assert_array_equal(O.round_bf16(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, 1 + 2.0 ** -8 + 2.0 ** -20])),
+                                  [1.0, 1 + 2.0 ** -6, 1 + 2.0 ** -7])
+
+
+def test_bf16_storage_mode_rounds_only_what_is_stored():
+    """With act_dtype = "bf16" the K/V a pass returns are exact bf16 values, the results move by the
+    size of bf16 rounding noise and no more, and the default mode is untouched."""
+    from dataclasses import replace
+    from tests.helpers import make_model, oracle_cfg, prompt_ids
+    sh, wt = make_model("tiny")
+    cfg = oracle_cfg(sh)
+    w = O.weights_to_f64(wt)
+    ids = prompt_ids(sh, 24)
+    a = O.causal_forward(cfg, w, ids)
+    b = O.causal_forward(replace(cfg, act_dtype="bf16"), w, ids)
+    c = O.causal_forward(replace(cfg, act_dtype="f64"), w, ids)
+    np.testing.assert_array_equal(a.logits, c.logits)
+    for l in range(cfg.n_layers):
+        np.testing.assert_array_equal(b.k_new[l], O.round_bf16(b.k_new[l]))
+        np.testing.assert_array_equal(b.v_new[l], O.round_bf16(b.v_new[l]))
+        assert not np.array_equal(a.k_new[l], O.round_bf16(a.k_new[l]))
+    d = np.abs(a.logits - b.logits).max()
+    assert 1e-5 < d < 3e-2, d
+    np.testing.assert_array_equal(a.hidden[0], b.hidden[0])        # the embedding rows are not an activation store
