@@ -7,16 +7,21 @@
  * forward over k*(k+1) token slots per sequence (paper, Section 3.3 footnote):
  * the k tokens proposed by the previous step, encoded causally against the
  * exact KV cache, plus k blocks of k mask tokens that pre-draft the next block
- * for every possible acceptance outcome (paper, Section 1 "three sections",
- * Section 3.2, figure "TiDAR Architecture").  After the forward the step keeps
- * the longest prefix of drafts that agree with the autoregressive prediction,
- * picks the pre-draft that matches that outcome and commits only the accepted
- * tokens' KV (Section 3.2; Section 3.3 "evict the KV cache").
+ * for every possible acceptance outcome (paper, Section 1, the description of
+ * what one generation step carries; Section 3.2; figure "TiDAR Architecture").
+ * After the forward the step keeps the longest prefix of drafts that agree with
+ * the autoregressive prediction, picks the pre-draft that matches that outcome
+ * and commits only the accepted tokens' KV (Section 3.2; Section 3.3, where the
+ * KV of rejected tokens is dropped).
  *
  * Conventions
- *   - Every entry point returns TIDAR_OK (0) or a negative TIDAR_E* code and
- *     leaves the context unchanged on error.  Nothing throws, aborts or traps.
- *     tidar_last_error() gives a human-readable message for the last failure.
+ *   - Every entry point returns TIDAR_OK (0) or a negative TIDAR_E* code.  Errors
+ *     found on the host (EINVAL, ECAPACITY, ENOMEM) are reported before anything
+ *     is launched and leave the context unchanged.  TIDAR_EDEVICE_TIMEOUT is
+ *     different: a kernel's bounded wait ran out, the pass's results are invalid
+ *     and the sequences it touched are released (they must be prefilled again).
+ *     Nothing throws, aborts or traps.  tidar_last_error() gives a
+ *     human-readable message for the last failure.
  *   - "host" / "device" on a pointer says where the memory lives.
  *   - Weights and the arena are BORROWED: the caller allocates them (for
  *     instance through PyTorch), keeps them alive until tidar_free and must
@@ -55,7 +60,11 @@ typedef struct {
   int32_t max_batch;        /* sequences a context can hold and step together              */
   int32_t max_seq_len;      /* per sequence; a step needs n + 2k <= max_seq_len            */
   int32_t page_size;        /* KV page length in tokens (64)                               */
-  float   beta;             /* verification mix (Section 4.4.3); only 1.0 is implemented   */
+  float   beta;             /* verification mix in [0, 1] (paper Section 4.4.3): a draft is checked
+                               against argmax(beta * logits_ar + (1 - beta) * logits_diff).
+                               1.0 (verification by the autoregressive prediction alone) is
+                               the hot path and makes greedy TiDAR equal greedy AR decoding;
+                               below 1 every verified position costs one more LM-head row  */
   float   temperature;      /* 0 = greedy; only greedy is implemented                      */
   uint64_t sample_seed;     /* reserved for seeded sampling                                */
   int32_t debug;            /* bit 0: keep per-layer hidden states and full logits of the
@@ -99,15 +108,19 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *weights,
                void *arena /*device*/, size_t arena_bytes, void *cuda_stream, tidar_ctx **out);
 
 /* First pass for sequence slot `seq` (0 <= seq < max_batch), replacing whatever the
- * slot held (paper, Section 3.2 "In the start of the generation"; Appendix B): the
- * prompt is encoded causally and its KV cached; one block of k mask tokens is
+ * slot held (paper, Section 3.2, how generation begins; Appendix B, the prefill mask):
+ * the prompt is encoded causally and its KV cached; one block of k mask tokens is
  * appended with bidirectional attention.  Emits the first settled token (argmax of
  * the last prompt row) to *out_first_token and stores the first draft block.
  * Needs 1 <= n_prompt, 1 <= k <= k_max, n_prompt + 2k <= max_seq_len.             */
 int tidar_prefill(tidar_ctx *ctx, int32_t seq, const int32_t *prompt_ids /*host*/, int32_t n_prompt,
                   int32_t k, int32_t *out_first_token /*host*/);
 
-/* One decode step for the listed sequences (all prefetched with the same k).
+/* One decode step for the listed sequences (all prefilled with the same k): paper,
+ * Section 3.2 (verify the previous step's drafts against the autoregressive predictions
+ * of the same pass, keep the longest agreeing prefix, hand the matching pre-draft to the
+ * next step) with the slot layout of the Section 3.3 footnote and the attention mask of
+ * figure "TiDAR Attention Masks".
  * forced_accept: NULL, or per sequence 0 = natural acceptance, L in [1,k] = accept
  * exactly L slots whatever the drafts were (benchmark hook; not in the paper).
  * On return out_n[i] = L_i and out_tokens[i*k_max .. i*k_max+L_i) = the L_i new tokens:
@@ -124,6 +137,38 @@ int tidar_step(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_
  * length to check capacity without reading the device).                           */
 int tidar_step_async(tidar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, const int32_t *forced_accept);
 int tidar_step_wait(tidar_ctx *ctx, int32_t *out_tokens /*host,[n_seqs][k_max]*/, int32_t *out_n /*host*/);
+
+/* A decode step with a block length chosen for this step (paper Section 5: the block length
+ * can follow the compute profile; with B sequences the step has B*k*(k+1) token slots, and
+ * those are "free" only while the pass stays memory-bound).  1 <= k <= k_max.  The step uses
+ * the first k entries of each sequence's block; where a sequence holds fewer drafts than k
+ * (its previous pass ran a shorter block, or it was an autoregressive step) the missing drafts
+ * are fed as mask tokens and are never accepted, so such a step emits fewer tokens but leaves a
+ * full block of k behind.  Everything else as tidar_step.                                 */
+int tidar_step_k(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs, int32_t k,
+                 const int32_t *forced_accept /*host or NULL*/, int32_t *out_tokens /*host,[n_seqs][k_max]*/,
+                 int32_t *out_n /*host,[n_seqs]*/);
+
+/* The block length that keeps a step of n_seqs sequences within row_budget token slots:
+ * the largest k <= k_max with n_seqs*k*(k+1) <= row_budget (at least 1).  row_budget <= 0
+ * selects 288, one row block of the projection kernels, about where the 8B-class step
+ * leaves the memory-bound region on a B200 (measured ridge: 220 .. 288 rows).  Host only. */
+int tidar_ridge_k(const tidar_ctx *ctx, int32_t n_seqs, int32_t row_budget);
+
+/* One plain autoregressive step (paper Section 3.1: the model keeps a causal, chain-factorised
+ * mode): a single causal slot per sequence, the settled token at position n, no mask slots.
+ * Emits exactly one token per sequence (out_tokens[i]) and leaves a block that holds that
+ * token alone, so a later tidar_step_k finds no drafts and accepts one token on its first
+ * pass.  The baseline the paper's speed-ups are quoted against (Section 4.3).             */
+int tidar_ar_step(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs, int32_t *out_tokens /*host,[n_seqs]*/);
+
+/* Likelihood scoring in the autoregressive mode (paper Section 3.1, the chain-factorised joint
+ * distribution; Section 4.2, likelihood tasks): one causal pass over ids[0..n) and
+ * logprobs[i] = log softmax(logits at position i)[ids[i+1]] for i in [0, n-1).
+ * Uses sequence slot `seq` as scratch: whatever it held is dropped and the slot is left
+ * empty.  The log-sum-exp runs over vocabulary chunks; full logits are never kept.
+ * Needs 2 <= n <= max_seq_len.  Synchronises the stream.                                  */
+int tidar_score(tidar_ctx *ctx, int32_t seq, const int32_t *ids /*host,[n]*/, int32_t n, float *logprobs /*host,[n-1]*/);
 
 /* Release the context (host state only; arena and weights belong to the caller). */
 int tidar_free(tidar_ctx *ctx);
@@ -144,8 +189,9 @@ int64_t tidar_launch_count(const tidar_ctx *ctx);
 int tidar_debug_set_block(tidar_ctx *ctx, int32_t seq, const int32_t *block /*host,[k]*/);
 int tidar_debug_get_block(tidar_ctx *ctx, int32_t seq, int32_t *block /*host,[k]*/);
 /* Results of the last pass; need cfg.debug bit 0.  Row r of a decode step is slot
- * r % (k*(k+1)) of the (r / (k*(k+1)))-th listed sequence; for a prefill the rows are
- * the last chunk's rows (see tidar_debug_last_rows).                               */
+ * r % (k*(k+1)) of the (r / (k*(k+1)))-th listed sequence; with beta < 1 the rows that mix
+ * causal slot j with the first slot of block j follow all slots (k per sequence).  For a
+ * prefill the rows are the last chunk's rows (see tidar_debug_last_rows).            */
 int tidar_debug_last_rows(const tidar_ctx *ctx, int32_t *n_rows, int32_t *first_row_position);
 int tidar_debug_get_logits(tidar_ctx *ctx, int32_t row0, int32_t n_rows, float *out /*host,[n_rows][vocab]*/);
 /* layer in [0, n_layers]: input of that layer; n_layers = input of the final norm. */
@@ -167,10 +213,35 @@ int tidar_debug_get_kv(tidar_ctx *ctx, int32_t seq, int32_t layer, int32_t pos0,
 #define TIDAR_TC_VERIFY  6
 #define TIDAR_TC_COUNT   7
 int tidar_debug_set_timing(tidar_ctx *ctx, int32_t on);
+/* Skipped-tile evidence for the attention kernel.  While `on`, every CTA of the tensor-core
+ * attention kernel adds the number of 64-key tiles it visits to a device counter.  Each call
+ * returns the count accumulated since the previous call in *visited (may be NULL), clears it
+ * and sets the switch.  Synchronises the stream.  A dense mask would visit, per 128-row query
+ * tile and KV head, every 64-key tile of [cache | step slots].                          */
+int tidar_debug_count_attention_tiles(tidar_ctx *ctx, int32_t on, uint64_t *visited /*host*/);
+/* In-kernel timeline of a decode step, for the launch mode the benchmark times (replayed
+ * graph, programmatic launches), where events cannot be put between kernels without changing
+ * the schedule.  While enabled, every kernel of a step records, in two device words of its
+ * own, the earliest moment one of its CTAs got past the dependency on the previous kernel and
+ * the latest moment one finished (%globaltimer).  After the step, class_ms[cls] is the sum of
+ * (end - start) over the launches of a class (TIDAR_TC_*), *busy_ms the sum over all launches
+ * and *span_ms the time from the first start to the last end.  Costs two atomics per CTA;
+ * switching it on or off re-captures the step's graph.  impl 0 only.                    */
+int tidar_debug_set_timeline(tidar_ctx *ctx, int32_t on);
+int tidar_debug_get_timeline(tidar_ctx *ctx, float *class_ms /*host,[TIDAR_TC_COUNT]*/, float *busy_ms /*host, or NULL*/,
+                             float *span_ms /*host, or NULL*/);
+/* Test hook for the error plumbing: writes `value` into the device status word that the
+ * kernels set when a bounded wait gives up.  The next tidar_step / tidar_prefill /
+ * tidar_sync then reports TIDAR_EDEVICE_TIMEOUT exactly as after a real timeout.  No
+ * kernel is made to wait.                                                             */
+int tidar_debug_force_status(tidar_ctx *ctx, int32_t value);
 int tidar_debug_get_timing(tidar_ctx *ctx, float *ms /*host,[TIDAR_TC_COUNT]*/);
 
 /* ---- structured-mask attention alone (microbenchmark and unit parity) -------------
- * Runs the step's attention kernel on caller-provided tensors (all DEVICE, bf16):
+ * The attention of one decode step under the mask of the paper's figure "TiDAR Attention
+ * Masks" (Section 3.1: drafted tokens causal, each mask block bidirectional within itself
+ * and blind to the other blocks), on caller-provided tensors (all DEVICE, bf16, 16-byte
+ * aligned):
  *   q        [n_seqs*T][n_q_heads][head_dim], T = k*(k+1), slot order of a decode step
  *   k_pages, v_pages : page pools [n_pages][n_kv_heads][page_size][head_dim]; the
  *              cached prefix AND the k causal slots of the step (positions n..n+k-1)
@@ -181,7 +252,10 @@ int tidar_debug_get_timing(tidar_ctx *ctx, float *ms /*host,[TIDAR_TC_COUNT]*/);
  *   out      [n_seqs*T][n_q_heads*head_dim]
  * Mask per the decode-step definition: causal slot j sees positions < n+j+1; mask
  * slot (b,i) sees positions < n+b+1 plus the k local slots of block b.
- * Uses ctx only for its stream, kernel implementation choice and scratch.          */
+ * seq_len values are clamped to [0, pages_per_seq*page_size - k]; page indices outside
+ * [0, n_pages) contribute nothing (impl 1) or zeros (impl 0: out-of-range tiles load as 0).
+ * Uses ctx only for its stream, kernel implementation choice and scratch.
+ * Errors: EINVAL (null or misaligned pointer, row capacity), ECUDA.                  */
 int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const void *v_pages,
                     int32_t n_pages, const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
                     const void *k_local, const void *v_local, void *out,
@@ -200,31 +274,42 @@ int tidar_gemm(tidar_ctx *ctx, const void *A, const void *W, int32_t R, int32_t 
                int32_t splits, float *out);
 
 /* Wait for everything enqueued on the context's stream and report a device-side
- * timeout (TIDAR_EDEVICE_TIMEOUT) if a kernel's bounded wait gave up.                  */
+ * timeout (TIDAR_EDEVICE_TIMEOUT) if a kernel's bounded wait gave up (results of the
+ * calls since the last check are then invalid).                                        */
 int tidar_sync(tidar_ctx *ctx);
 
 /* ---- structured-mask attention for callers that cannot allocate ---------------------
  * (The paper has no counterpart: this is a packaging variant of tidar_attention.)
- * Same computation, same tensor layouts and same mask as tidar_attention, but it needs
- * no context and no arena: the shapes come as plain arguments and the per-row
- * visibility table, which tidar_attention keeps in the caller-allocated arena, lives in
- * a fixed table built into the library image.  It is meant for hosts that hold device
- * tensors but may not call an allocator where they need attention: a server whose
- * memory pool belongs wholly to another component, a latency-critical loop (cudaMalloc
- * may stall every stream of the device), a plug-in that is handed buffers only.
+ * Same mask, same tensor layouts and the same result (within rounding) as
+ * tidar_attention, but it needs no context and no arena: the shapes come as plain
+ * arguments and the per-row visibility table, which tidar_attention keeps in the
+ * caller-allocated arena, lives in a fixed table built into the library image.  It is
+ * meant for hosts that hold device tensors but may not call an allocator where they need
+ * attention: a server whose memory pool belongs wholly to another component, a loop that
+ * must not enter the allocator (cudaMalloc may stall every stream of the device), a
+ * plug-in that is handed buffers only.
  * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   - It always runs the plain CUDA-core kernel (one warp per row and query head, fp32
+ *     accumulation, K/V re-read once per query head, no tile skipping), not the
+ *     tensor-core kernel: correct and allocation-free, not fast (about 30 times slower
+ *     than tidar_attention with impl 0 at a thousand cached positions).
  *   - Limit: n_seqs * k * (k+1) <= 4352 rows (16 sequences at k = 16); beyond that the
  *     call returns TIDAR_ECAPACITY and launches nothing.  page_size is 64.
  *   - Each GPU that loads the library holds the table (85 KiB) until the process exits.
  *   - The first call on a device looks up the table's device address (with that device
- *     current); make that first call outside any stream capture.
+ *     current); make that first call outside any stream capture.  The look-up is not
+ *     synchronised between host threads: concurrent first calls are harmless (they store
+ *     the same address) but not ordered.
  *   - All calls on one device share the table and each call rewrites the entries it uses,
  *     so nothing needs clearing; but two calls whose kernels may overlap on the GPU
  *     (different streams, no ordering between them) race on it.  Serialise them.
  *   - Work is enqueued on cuda_stream (a cudaStream_t, NULL = default) of the current
- *     device; the call does not synchronise.  All data pointers are DEVICE pointers.
+ *     device; the call does not synchronise.  All data pointers are DEVICE pointers,
+ *     16-byte aligned (page_table, seq_len: 4-byte).  seq_len values are clamped to
+ *     [0, pages_per_seq*64 - k]; keys on pages outside [0, n_pages) are skipped; a row
+ *     left without any visible key gets zeros.
  * Errors: TIDAR_EINVAL, TIDAR_ECAPACITY, TIDAR_ECUDA; message via tidar_last_error(NULL). */
-int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages,
+int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages, int32_t n_pages,
                            const int32_t *page_table, int32_t pages_per_seq, const int32_t *seq_len,
                            const void *k_local, const void *v_local, void *out,
                            int32_t n_seqs, int32_t k, int32_t n_q_heads, int32_t n_kv_heads,

@@ -64,6 +64,10 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_step": (C.c_int, [ctxp, P(I32), I32, P(I32), P(I32), P(I32)]),
         "tidar_step_async": (C.c_int, [ctxp, P(I32), I32, P(I32)]),
         "tidar_step_wait": (C.c_int, [ctxp, P(I32), P(I32)]),
+        "tidar_step_k": (C.c_int, [ctxp, P(I32), I32, I32, P(I32), P(I32), P(I32)]),
+        "tidar_ar_step": (C.c_int, [ctxp, P(I32), I32, P(I32)]),
+        "tidar_ridge_k": (C.c_int, [ctxp, I32, I32]),
+        "tidar_score": (C.c_int, [ctxp, I32, P(I32), I32, P(C.c_float)]),
         "tidar_free": (C.c_int, [ctxp]),
         "tidar_last_error": (C.c_char_p, [ctxp]),
         "tidar_seq_len": (C.c_int, [ctxp, I32]),
@@ -80,7 +84,11 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_attention": (C.c_int, [ctxp, VP, VP, VP, I32, VP, I32, VP, VP, VP, VP, I32, I32]),
         "tidar_gemm": (C.c_int, [ctxp, VP, VP, I32, I32, I32, I32, VP]),
         "tidar_sync": (C.c_int, [ctxp]),
-        "tidar_attention_static": (C.c_int, [VP, VP, VP, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
+        "tidar_attention_static": (C.c_int, [VP, VP, VP, I32, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
+        "tidar_debug_force_status": (C.c_int, [ctxp, I32]),
+        "tidar_debug_count_attention_tiles": (C.c_int, [ctxp, I32, P(C.c_uint64)]),
+        "tidar_debug_set_timeline": (C.c_int, [ctxp, I32]),
+        "tidar_debug_get_timeline": (C.c_int, [ctxp, P(C.c_float), P(C.c_float), P(C.c_float)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -122,7 +130,8 @@ class Tidar:
     """One library context: model weights + KV arena on one GPU."""
 
     def __init__(self, shape, packed: dict, k_max: int, max_batch: int = 1, max_seq_len: int = 4096,
-                 debug: int = 0, impl: int = 0, device="cuda:0", stream: Optional[torch.cuda.Stream] = None):
+                 debug: int = 0, impl: int = 0, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
+                 guard_bytes: int = 0, beta: float = 1.0):
         self.lib = load()
         self.shape, self.k_max, self.max_batch = shape, k_max, max_batch
         self.device = torch.device(device)
@@ -130,16 +139,22 @@ class Tidar:
             n_layers=len(packed["layers"]), d_model=shape.d_model, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
             head_dim=shape.head_dim, d_ffn=shape.d_ffn, vocab=shape.vocab, tie_lm_head=int(shape.tie_lm_head),
             rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, mask_token_id=shape.mask_token_id, k_max=k_max,
-            max_batch=max_batch, max_seq_len=max_seq_len, page_size=64, beta=1.0, temperature=0.0, sample_seed=0,
+            max_batch=max_batch, max_seq_len=max_seq_len, page_size=64, beta=beta, temperature=0.0, sample_seed=0,
             debug=debug, impl=impl)
         self.cfg = cfg
         nbytes = C.c_size_t(0)
         rc = self.lib.tidar_arena_bytes(C.byref(cfg), C.byref(nbytes))
         if rc:
             raise TidarError(rc, (self.lib.tidar_last_error(None) or b"").decode())
+        # guard_bytes > 0: a sentinel-filled tail right behind the arena (the library is told
+        # nothing about it), so that a write past the arena can be detected: arena_guard_intact()
+        self._guard_bytes = int(guard_bytes)
         with torch.cuda.device(self.device):
-            self.arena = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+            self.arena = torch.empty(nbytes.value + 256 + self._guard_bytes, dtype=torch.uint8, device=self.device)
         base = (self.arena.data_ptr() + 255) // 256 * 256
+        self._guard_off = base - self.arena.data_ptr() + nbytes.value
+        if self._guard_bytes:
+            self.arena[self._guard_off:].fill_(0xA5)
         self._packed = packed                     # keep the borrowed tensors alive
         nl = len(packed["layers"])
         arrs = {}
@@ -163,6 +178,13 @@ class Tidar:
     def _check(self, rc: int):
         if rc:
             raise TidarError(rc, (self.lib.tidar_last_error(self.ctx) or b"").decode())
+
+    def arena_guard_intact(self) -> bool:
+        """True if nothing wrote into the sentinel tail behind the arena (guard_bytes > 0)."""
+        if not self._guard_bytes:
+            return True
+        torch.cuda.synchronize(self.device)
+        return bool((self.arena[self._guard_off:] == 0xA5).all())
 
     def close(self):
         if getattr(self, "ctx", None):
@@ -189,6 +211,32 @@ class Tidar:
         n = np.empty(len(s), dtype=np.int32)
         self._check(self.lib.tidar_step(self.ctx, _ip(s), len(s), _ip(f) if f is not None else None, _ip(toks), _ip(n)))
         return [toks[i, :n[i]].tolist() for i in range(len(s))], n.tolist()
+
+    def step_k(self, seqs: Sequence[int], k: int, forced: Optional[Sequence[int]] = None):
+        """A decode step with block length k chosen for this step (see tidar_step_k)."""
+        s = _i32(seqs)
+        f = _i32(forced) if forced is not None else None
+        toks = np.empty((len(s), self.k_max), dtype=np.int32)
+        n = np.empty(len(s), dtype=np.int32)
+        self._check(self.lib.tidar_step_k(self.ctx, _ip(s), len(s), k, _ip(f) if f is not None else None, _ip(toks), _ip(n)))
+        return [toks[i, :n[i]].tolist() for i in range(len(s))], n.tolist()
+
+    def ar_step(self, seqs: Sequence[int]) -> List[int]:
+        """One plain autoregressive step: one new token per sequence (see tidar_ar_step)."""
+        s = _i32(seqs)
+        out = np.empty(len(s), dtype=np.int32)
+        self._check(self.lib.tidar_ar_step(self.ctx, _ip(s), len(s), _ip(out)))
+        return out.tolist()
+
+    def ridge_k(self, n_seqs: int, row_budget: int = 0) -> int:
+        return int(self.lib.tidar_ridge_k(self.ctx, n_seqs, row_budget))
+
+    def score(self, seq: int, ids: Sequence[int]) -> np.ndarray:
+        """log p(ids[i+1] | ids[..i]) for i in [0, n-1) from one causal pass (see tidar_score)."""
+        a = _i32(ids)
+        out = np.empty(len(a) - 1, dtype=np.float32)
+        self._check(self.lib.tidar_score(self.ctx, seq, _ip(a), len(a), out.ctypes.data_as(C.POINTER(C.c_float))))
+        return out
 
     def step_async(self, seqs: Sequence[int], forced: Sequence[int]):
         s, f = _i32(seqs), _i32(forced)
@@ -248,6 +296,28 @@ class Tidar:
         self._check(self.lib.tidar_debug_get_kv(self.ctx, seq, layer, pos0, npos, k.ctypes.data_as(P16), v.ctypes.data_as(P16)))
         return k, v
 
+    def force_status(self, value: int):
+        """Test hook: pretend a kernel's bounded wait gave up (see tidar_debug_force_status)."""
+        self._check(self.lib.tidar_debug_force_status(self.ctx, int(value)))
+
+    def count_attention_tiles(self, on: bool) -> int:
+        """Key tiles the attention kernel visited since the last call; sets the counter's switch."""
+        v = C.c_uint64(0)
+        self._check(self.lib.tidar_debug_count_attention_tiles(self.ctx, int(on), C.byref(v)))
+        return int(v.value)
+
+    def set_timeline(self, on: bool):
+        self._check(self.lib.tidar_debug_set_timeline(self.ctx, int(on)))
+
+    def timeline(self) -> dict:
+        """Per-class kernel time (ms) of the last step from in-kernel stamps, plus 'busy' and 'span'."""
+        ms = (C.c_float * len(TC_NAMES))()
+        busy, span = C.c_float(0), C.c_float(0)
+        self._check(self.lib.tidar_debug_get_timeline(self.ctx, ms, C.byref(busy), C.byref(span)))
+        out = {n: float(ms[i]) for i, n in enumerate(TC_NAMES)}
+        out["busy"], out["span"] = float(busy.value), float(span.value)
+        return out
+
     def set_timing(self, on: bool):
         self._check(self.lib.tidar_debug_set_timing(self.ctx, int(on)))
 
@@ -281,7 +351,7 @@ def attention_static(q, k_pages, v_pages, page_table, seq_len, k_local, v_local,
     (``n_seqs * k * (k+1)``); calls that may overlap on the GPU must be serialised.
     """
     lib = load()
-    rc = lib.tidar_attention_static(q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), page_table.data_ptr(),
+    rc = lib.tidar_attention_static(q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), k_pages.shape[0], page_table.data_ptr(),
                                     page_table.shape[1], seq_len.data_ptr(), k_local.data_ptr(), v_local.data_ptr(),
                                     out.data_ptr(), n_seqs, k, n_q_heads, n_kv_heads, head_dim,
                                     C.c_void_p(stream.cuda_stream if stream is not None else 0))

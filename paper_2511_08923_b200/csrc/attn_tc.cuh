@@ -48,6 +48,7 @@ struct Args {
   float *part_O;                             // [splits][R][Hq][hd]  (splits > 1)
   float *part_ml;                            // [splits][R][Hq][2]
   int *status;
+  unsigned long long *tile_count;            // diagnostics: += key tiles this CTA visits (null = off)
 };
 
 // Shared memory of one CTA; everything is dynamic so that the 1024-byte alignment the
@@ -77,7 +78,7 @@ static_assert(sizeof(Ctl) <= 256, "control block must fit its slot");
 template <int HD>
 __global__ void __launch_bounds__(THREADS, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-               const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a) {
+               const __grid_constant__ CUtensorMap tmKloc, const __grid_constant__ CUtensorMap tmVloc, const Args a, const TlSlot tl) {
   using L = Smem<HD>;
   constexpr int NH = L::NH;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -117,6 +118,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   }
   __syncthreads();
   pdl_wait();                 // everything below reads what earlier kernels of the pass wrote
+  if (threadIdx.x == 0) tl_go(tl);
 
   // ---- per-row metadata (softmax threads own one MMA row each) and the tile's key range ----
   const int my_row = (warp & 3) * 32 + lane;             // MMA row = TMEM lane (softmax warps only)
@@ -145,6 +147,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   const int nt = t_end - t_begin;
   const int seq = row0 < a.R ? a.seq[row0] : 0;
   volatile int *abortp = &ctl.abort_flag;
+  if (threadIdx.x == 0 && a.tile_count) atomicAdd(a.tile_count, (unsigned long long)nt);
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -382,20 +385,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     sm100::tc_fence_after();
     sm100::tmem_dealloc(tmem, L::TMEM_COLS);
   }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // Merge the per-split partial results: O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
 // HD / 4 threads per (row, head), four consecutive columns each: 16-byte loads, 8-byte stores.
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_O, const float *__restrict__ part_ml, int splits, int R, int Hq,
-                               bf16 *__restrict__ O) {
+                               bf16 *__restrict__ O, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   constexpr int PER = HD / 4;
   const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t wid = gid / PER;
   const int c4 = (int)(gid % PER);
-  if (wid >= (size_t)R * Hq) return;
+  if (wid >= (size_t)R * Hq) { if (threadIdx.x == 0) tl_end(tl); return; }
   float M = -INFINITY;
   for (int s = 0; s < splits; ++s) M = fmaxf(M, part_ml[((size_t)s * R * Hq + wid) * 2]);
   float den = 0.f;
@@ -412,6 +417,7 @@ __global__ void attn_combine_kernel(const float *__restrict__ part_O, const floa
   __nv_bfloat162 h0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
   uint2 u; u.x = *reinterpret_cast<uint32_t *>(&h0); u.y = *reinterpret_cast<uint32_t *>(&h1);
   reinterpret_cast<uint2 *>(O + wid * HD)[c4] = u;
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 }  // namespace attn_tc

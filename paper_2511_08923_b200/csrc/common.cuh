@@ -27,6 +27,7 @@ struct RowMeta {
 struct KvGeom {
   int32_t n_kv_heads, head_dim, page_size, pages_per_seq;
   const int32_t *page_table;   // [max_batch][pages_per_seq]
+  int32_t n_pages;             // pages in the pool; 0 = the table is the library's own and needs no check
 };
 
 __device__ __forceinline__ size_t kv_row_offset(const KvGeom &g, int seq, int position, int kvh) {
@@ -53,3 +54,18 @@ __device__ __forceinline__ float warp_max(float v) {
 // be scheduled early in the same way.  Both are no-ops in a plain launch.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Optional in-kernel timeline (diagnostics; off when t is null).  Every launch of a pass gets a
+// slot of two words, both zeroed before the pass: t[0] collects the bit-wise complement of the
+// EARLIEST moment a CTA got past its dependency on the previous kernel (atomicMax of ~time =
+// minimum of time), t[1] the LATEST moment a CTA finished.  end - start is then the time the
+// launch really occupied inside a replayed graph with programmatic launches, where events
+// cannot be placed without changing the schedule.  One thread per CTA calls each.
+struct TlSlot { unsigned long long *t; };
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void tl_go(TlSlot s) { if (s.t) atomicMax(s.t, ~global_ns()); }
+__device__ __forceinline__ void tl_end(TlSlot s) { if (s.t) atomicMax(s.t + 1, global_ns()); }

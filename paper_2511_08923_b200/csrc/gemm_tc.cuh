@@ -84,7 +84,7 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(
 
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const Args g, const TlSlot tl) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t w_full[8], w_empty[8], a_full[8], a_empty[8], tmem_full_bar, tmem_empty_bar;
   __shared__ uint32_t tmem_base_slot;
@@ -154,6 +154,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint64_t pol_a = sm100::policy_evict_last();
       int s = 0; uint32_t ph = 0; bool ok = true;
       pdl_wait();                      // the activations are the previous kernel's output
+      tl_go(tl);
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item w = decode_item(g, item);
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
@@ -466,6 +467,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     sm100::tc_fence_after();
     sm100::tmem_dealloc(tmem_acc, TMEM_COLS);
   }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // ---- host side ----------------------------------------------------------------------

@@ -25,26 +25,33 @@ __device__ __forceinline__ void embed_row_to_f32(const bf16 *__restrict__ e, flo
 
 // ---------------------------------------------------------------------------
 // Slot assembly + embedding gather for a decode step.
-// Slot layout per sequence (k causal slots, then k blocks of k mask slots;
+// Slot layout per sequence (k causal slots, then n_blocks blocks of k mask slots;
 // paper Section 3.3 footnote, figure "TiDAR Attention Masks"):
 //   causal j       : token block[j], position n+j
 //   mask (b, i)    : [MASK], position n+b+1+i (no label shift: a mask slot predicts
 //                    its own position; paper Section 4.4.3)
+// n_blocks = k for a TiDAR step; n_blocks = 0 for a plain autoregressive step (the
+// causal section alone: paper Section 3.1, the model keeps its autoregressive mode).
+// The step may use a block length k that differs from the one the previous pass left
+// (blk_len[seq] valid entries): drafts the sequence does not have are fed as [MASK]
+// and can never be accepted (see verify_select_kernel).
 // One block per row; also snapshots n into step_n for the commit kernel.
 // ---------------------------------------------------------------------------
 __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ seq_len,
-                                     const int32_t *__restrict__ block_ids, int k, int k_max, int mask_id,
+                                     const int32_t *__restrict__ block_ids, const int32_t *__restrict__ blk_len, int k, int n_blocks,
+                                     int k_max, int mask_id,
                                      int32_t *__restrict__ step_n, const bf16 *__restrict__ embed, int d,
-                                     float *__restrict__ X) {
+                                     float *__restrict__ X, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
-  const int T = k * (k + 1);
+  if (threadIdx.x == 0) tl_go(tl);
+  const int T = k * (n_blocks + 1);
   const int r = blockIdx.x;
   const int s = r / T, slot = r % T;
   const int seq = step_seqs[s];
   const int n = seq_len[seq];
   int id;
-  if (slot < k) id = block_ids[seq * k_max + slot]; else id = mask_id;
+  if (slot < k && slot < blk_len[seq]) id = block_ids[seq * k_max + slot]; else id = mask_id;
   if (threadIdx.x == 0) {
     if (slot == 0) step_n[s] = n;
     m.seq[r] = seq;
@@ -59,6 +66,7 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
     }
   }
   embed_row_to_f32(embed + (size_t)id * d, X + (size_t)r * d, d);
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // Prefill chunk: rows g = row0 .. row0+rows-1 of [prompt ; k mask tokens]
@@ -82,12 +90,14 @@ __global__ void assemble_prefill_kernel(RowMeta m, int seq, int row0, int n_prom
 }
 
 // Row metadata for the stand-alone attention entry point (same slot layout as a step).
-__global__ void attn_meta_kernel(RowMeta m, const int32_t *__restrict__ seq_len, int k, int R) {
+// seq_len comes from the caller: it is clamped to [0, n_max] (n_max = the positions the page
+// table can back minus the k causal slots), so that no row looks past the table.
+__global__ void attn_meta_kernel(RowMeta m, const int32_t *__restrict__ seq_len, int k, int R, int n_max) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= R) return;
   const int T = k * (k + 1);
   const int s = r / T, slot = r % T;
-  const int n = seq_len[s];
+  const int n = min(max(seq_len[s], 0), n_max);
   m.seq[r] = s;
   if (slot < k) {
     m.pos[r] = n + slot; m.nvis[r] = n + slot + 1; m.loc0[r] = 0; m.nloc[r] = 0;
@@ -100,16 +110,18 @@ __global__ void attn_meta_kernel(RowMeta m, const int32_t *__restrict__ seq_len,
 // cos/sin of pos * theta^(-2i/hd), evaluated in double once per pass (shared by every
 // layer and head), stored as float.
 __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int R, int half, double theta,
-                                  float *__restrict__ cs, float *__restrict__ sn) {
+                                  float *__restrict__ cs, float *__restrict__ sn, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= R * half) return;
+  if (t >= R * half) { if (threadIdx.x == 0) tl_end(tl); return; }
   const int r = t / half, i = t % half;
   const double inv = pow(theta, -(double)i / (double)half);
   double s, c;
   sincos((double)pos[r] * inv, &s, &c);
   cs[t] = (float)c; sn[t] = (float)s;
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // ---------------------------------------------------------------------------
@@ -120,9 +132,10 @@ __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int R, int ha
 template <int THREADS, typename SLAB>
 __global__ void __launch_bounds__(THREADS)
 rmsnorm_reduce_kernel(float *__restrict__ X, const SLAB *__restrict__ partials, int S, size_t partial_stride,
-                      const bf16 *__restrict__ gain, float eps, int d, bf16 *__restrict__ A) {
+                      const bf16 *__restrict__ gain, float eps, int d, bf16 *__restrict__ A, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   extern __shared__ float row[];
   __shared__ float red[THREADS / 32];
   const int r = blockIdx.x;
@@ -153,6 +166,7 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const SLAB *__restrict__ partials, 
     uint2 ob; ob.x = *reinterpret_cast<uint32_t *>(&o0); ob.y = *reinterpret_cast<uint32_t *>(&o1);
     *reinterpret_cast<uint2 *>(A + (size_t)r * d + c) = ob;
   }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // ---------------------------------------------------------------------------
@@ -167,9 +181,10 @@ __global__ void __launch_bounds__(256)
 rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
                RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
                bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
-               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc) {
+               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   // a work unit is 4 consecutive dims i..i+3 of the first half of one
   // head together with their rotation partners i+hd/2..
   const int r = blockIdx.x, half = hd / 2, upr = half / 4;          // units per head
@@ -211,6 +226,7 @@ rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, 
     *reinterpret_cast<uint2 *>(dst + i) = o1;
     *reinterpret_cast<uint2 *>(dst + i + half) = o2;
   }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // SwiGLU on an fp32 [R][2*ffn] projection whose columns interleave (gate_f, up_f).
@@ -225,14 +241,15 @@ __global__ void swiglu_kernel(const float *__restrict__ GU, int R, int ffn, bf16
 // cover features [f0, f0 + nf): H[r][f0 + f] = silu(sum_s gate) * (sum_s up).  Two features per thread.
 template <typename SLAB>
 __global__ void swiglu_slab_kernel(const SLAB *__restrict__ slabs, int S, size_t stride, int R, int ld, int nf, int f0, int ldh,
-                                   bf16 *__restrict__ H) {
+                                   bf16 *__restrict__ H, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   // two features per thread; silu with the fast division of the fused epilogue (a precise
   // division costs ~170 cycles per result and was most of this kernel's time)
   const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int nf2 = nf / 2;
-  if (t >= (size_t)R * nf2) return;
+  if (t >= (size_t)R * nf2) { if (threadIdx.x == 0) tl_end(tl); return; }
   const int r = (int)(t / nf2), f = (int)(t % nf2) * 2;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);                      // gate f, up f, gate f+1, up f+1
   for (int s = 0; s < S; ++s) {
@@ -241,6 +258,7 @@ __global__ void swiglu_slab_kernel(const SLAB *__restrict__ slabs, int S, size_t
   }
   __nv_bfloat162 o = __floats2bfloat162_rn(__fdividef(acc.x, 1.f + __expf(-acc.x)) * acc.y, __fdividef(acc.z, 1.f + __expf(-acc.z)) * acc.w);
   *reinterpret_cast<__nv_bfloat162 *>(H + (size_t)r * ldh + f0 + f) = o;
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // Running per-row argmax over a chunk of logits [R][ncols] (fp32, leading dim ld)
@@ -281,11 +299,12 @@ __global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int nco
 // "nothing valid".  Lowest index wins ties, which makes the result independent of the
 // order in which candidates are combined.
 __global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t *__restrict__ pi, int G, int R,
-                                    float *__restrict__ best_val, int32_t *__restrict__ best_idx) {
+                                    float *__restrict__ best_val, int32_t *__restrict__ best_idx, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (r >= R) return;
+  if (r >= R) { if (threadIdx.x == 0) tl_end(tl); return; }
   float bv = -INFINITY; int bi = 0x7fffffff;
   for (int g = lane; g < G; g += 32) {
     const float v = pv[(size_t)r * G + g]; const int i = pi[(size_t)r * G + g];
@@ -297,6 +316,7 @@ __global__ void argmax_merge_kernel(const float *__restrict__ pv, const int32_t 
     if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
   }
   if (lane == 0) { best_val[r] = bv; best_idx[r] = bi == 0x7fffffff ? 0 : bi; }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // out[i] = sum over S slabs (fixed order) of in[s * stride + i].
@@ -309,53 +329,129 @@ __global__ void slab_sum_kernel(const float *__restrict__ in, int S, size_t stri
 }
 
 // ---------------------------------------------------------------------------
-// Draft / verify / select (paper Section 3.2; Section 4.4.3 with beta = 1).
+// Draft / verify / select (paper Section 3.2; Section 4.4.3).
 // One warp per sequence, lane i = causal slot i:
-//   target_i = argmax of causal slot i's logits (prediction for position n+i+1);
-//   draft i >= 1 agrees iff block[i] == target_{i-1};
+//   target_i = verified prediction for position n+i+1: argmax of causal slot i's logits, or
+//              (tgt_ids != null) the argmax of the row that mixes them with the first slot
+//              of block i;
+//   draft i >= 1 agrees iff the sequence had a draft there (i < blk_len) and
+//              block[i] == target_{i-1};
 //   L = 1 + length of the leading run of agreeing drafts (slot 0 is settled), or the
 //   forced value;  emitted = block[1..L-1], target_{L-1};
-//   next block = target_{L-1}, then the argmax of mask slots (L-1, 1..k-1).
+//   next block = target_{L-1}, then the argmax of mask slots (L-1, 1..k-1); with no mask
+//   blocks (plain autoregressive step, k = 1) the next block is target_0 alone.
 // ---------------------------------------------------------------------------
-__global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const int32_t *__restrict__ step_seqs,
-                                     const int32_t *__restrict__ forced, int k, int k_max,
-                                     int32_t *__restrict__ block_ids, int32_t *__restrict__ step_L,
-                                     int32_t *__restrict__ out /*[n_seqs][k_max+1]*/) {
+__global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const int32_t *__restrict__ tgt_ids,
+                                     const int32_t *__restrict__ step_seqs,
+                                     const int32_t *__restrict__ forced, int k, int n_blocks, int k_max,
+                                     int32_t *__restrict__ block_ids, int32_t *__restrict__ blk_len, int32_t *__restrict__ step_L,
+                                     int32_t *__restrict__ out /*[n_seqs][k_max+1]*/, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   const int s = blockIdx.x, lane = threadIdx.x;
-  const int T = k * (k + 1);
+  const int T = k * (n_blocks + 1);
   const int seq = step_seqs[s];
   const int32_t *ids = arg_ids + (size_t)s * T;
   int32_t *blk = block_ids + (size_t)seq * k_max;
-  const int tgt = lane < k ? ids[lane] : -1;
-  const int mine = lane < k ? blk[lane] : -2;
+  const int valid = blk_len[seq];
+  const int tgt = lane < k ? (tgt_ids ? tgt_ids[(size_t)s * k + lane] : ids[lane]) : -1;
+  const int mine = lane < k ? (lane < valid ? blk[lane] : -2) : -2;
   const int prev_tgt = __shfl_up_sync(0xffffffffu, tgt, 1);
-  const bool agree = lane == 0 || (lane < k && mine == prev_tgt);
+  const bool agree = lane == 0 || (lane < k && lane < valid && mine == prev_tgt);
   const unsigned bits = __ballot_sync(0xffffffffu, agree);
   int L = __ffs(~bits) - 1;            // leading run of ones; bit 0 is always set
   if (L > k || L < 0) L = k;           // all 32 lanes agreeing gives ffs(0) = 0
   const int f = forced ? forced[s] : 0;
   if (f > 0) L = f;
   const int t_last = __shfl_sync(0xffffffffu, tgt, L - 1);
-  const int next_draft = (lane >= 1 && lane < k) ? ids[k + (L - 1) * k + lane] : 0;
+  const int next_draft = (n_blocks > 0 && lane >= 1 && lane < k) ? ids[k + (L - 1) * k + lane] : 0;
   const int shifted = __shfl_down_sync(0xffffffffu, mine, 1);     // block[lane+1]
   __syncwarp();
   if (lane < k) {
     out[(size_t)s * (k_max + 1) + 1 + lane] = lane < L - 1 ? shifted : (lane == L - 1 ? t_last : -1);
     blk[lane] = lane == 0 ? t_last : next_draft;
   }
-  if (lane == 0) { out[(size_t)s * (k_max + 1)] = L; step_L[s] = L; }
+  if (lane == 0) { out[(size_t)s * (k_max + 1)] = L; step_L[s] = L; blk_len[seq] = n_blocks > 0 ? k : 1; tl_end(tl); }
+}
+
+// Verification by a mix of the autoregressive and the diffusion prediction (paper Section 4.4.3:
+// argmax(beta * logits_ar + (1 - beta) * logits_diff)).  Logits are linear in the final-normed
+// hidden row, so the mix is taken there: row dst = beta * row a + (1 - beta) * row b of the LM
+// head's input, one extra input row per verified position, and the LM head's argmax of that row
+// is the argmax of the mixed logits.  Block i handles pair i:
+//   a = a0 + (i / k) * a_seq + (i % k) * a_j,  b likewise,  dst = dst0 + i.
+__global__ void mix_rows_kernel(bf16 *__restrict__ A, int d, float beta, int k, int a0, int a_seq, int a_j, int b0, int b_seq, int b_j,
+                                int dst0, TlSlot tl) {
+  pdl_trigger();
+  pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
+  const int i = blockIdx.x, s = i / k, j = i % k;
+  const bf16 *ra = A + (size_t)(a0 + s * a_seq + j * a_j) * d, *rb = A + (size_t)(b0 + s * b_seq + j * b_j) * d;
+  bf16 *ro = A + (size_t)(dst0 + i) * d;
+  for (int c = threadIdx.x * 2; c < d; c += blockDim.x * 2) {
+    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(ra + c));
+    const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(rb + c));
+    *reinterpret_cast<__nv_bfloat162 *>(ro + c) = __floats2bfloat162_rn(beta * x.x + (1.f - beta) * y.x, beta * x.y + (1.f - beta) * y.y);
+  }
+  if (threadIdx.x == 0) tl_end(tl);
+}
+
+// Running log-sum-exp of a row over vocabulary chunks, and the logit of the row's target id.
+// L [R][ld] holds the logits of ids [col0, col0 + ncols).  (run_max, run_sum) is updated so that
+// log sum_v exp(logit_v) = run_max + log(run_sum) after the last chunk; fixed reduction order.
+__global__ void __launch_bounds__(256)
+score_chunk_kernel(const float *__restrict__ L, int ld, int ncols, int col0, int first, const int32_t *__restrict__ target,
+                   float *__restrict__ run_max, float *__restrict__ run_sum, float *__restrict__ tgt_logit) {
+  __shared__ float red[8];
+  __shared__ float bcast;
+  const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float *row = L + (size_t)r * ld;
+  float m = -INFINITY;
+  for (int c = threadIdx.x; c < ncols; c += 256) m = fmaxf(m, row[c]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = red[0];
+    for (int i = 1; i < 8; ++i) t = fmaxf(t, red[i]);
+    bcast = first ? t : fmaxf(t, run_max[r]);
+  }
+  __syncthreads();
+  const float M = bcast;
+  float sum = 0.f;
+  for (int c = threadIdx.x; c < ncols; c += 256) sum += __expf(row[c] - M);
+  sum = warp_sum(sum);
+  __syncthreads();
+  if (lane == 0) red[warp] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += red[i];
+    if (!first) t += run_sum[r] * __expf(run_max[r] - M);
+    run_max[r] = M; run_sum[r] = t;
+    const int tg = target[r] - col0;
+    if (tg >= 0 && tg < ncols) tgt_logit[r] = row[tg];
+  }
+}
+
+// logprob[r] = tgt_logit[r] - (run_max[r] + log(run_sum[r]))
+__global__ void score_finish_kernel(const float *__restrict__ run_max, const float *__restrict__ run_sum, const float *__restrict__ tgt_logit,
+                                    int R, float *__restrict__ logprob) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < R) logprob[r] = tgt_logit[r] - (run_max[r] + logf(run_sum[r]));
 }
 
 // First-pass finish: settled token = argmax of the last prompt row; drafts = argmax
 // of mask rows 1..k-1 (paper Section 3.2, start of generation).
-__global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int row_last_prompt, int k, int k_max, int seq,
-                                      int n_prompt, int32_t *__restrict__ block_ids, int32_t *__restrict__ seq_len,
-                                      int32_t *__restrict__ out) {
+// row_first: the row whose argmax is the settled token (the last prompt row, or the extra row that
+// mixes it with the first mask row when beta < 1).
+__global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int row_last_prompt, int row_first, int k, int k_max, int seq,
+                                      int n_prompt, int32_t *__restrict__ block_ids, int32_t *__restrict__ blk_len,
+                                      int32_t *__restrict__ seq_len, int32_t *__restrict__ out) {
   const int i = threadIdx.x;
-  if (i < k) block_ids[(size_t)seq * k_max + i] = i == 0 ? arg_ids[row_last_prompt] : arg_ids[row_last_prompt + 1 + i];
-  if (i == 0) { seq_len[seq] = n_prompt; out[0] = arg_ids[row_last_prompt]; }
+  if (i < k) block_ids[(size_t)seq * k_max + i] = i == 0 ? arg_ids[row_first] : arg_ids[row_last_prompt + 1 + i];
+  if (i == 0) { seq_len[seq] = n_prompt; blk_len[seq] = k; out[0] = arg_ids[row_first]; }
 }
 
 // ---------------------------------------------------------------------------
@@ -370,14 +466,15 @@ __global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int r
 // ---------------------------------------------------------------------------
 __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ step_n,
                                  const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, int poison,
-                                 KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride) {
+                                 KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) tl_go(tl);
   const int s = blockIdx.x, l = blockIdx.y;
   const int seq = step_seqs[s];
   const int n = step_n[s], L = step_L[s];
   if (l == 0 && threadIdx.x == 0) seq_len[seq] = n + L;
-  if (!poison) return;
+  if (!poison) { if (threadIdx.x == 0) tl_end(tl); return; }
   bf16 *Kp = kv_base + (size_t)(2 * l) * pool_stride, *Vp = Kp + pool_stride;
   const int per = g.n_kv_heads * g.head_dim;
   const bf16 nanv = __ushort_as_bfloat16((unsigned short)0x7f7f);
@@ -386,6 +483,7 @@ __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const in
     const size_t off = kv_row_offset(g, seq, p, kvh) + c;
     Kp[off] = nanv; Vp[off] = nanv;
   }
+  if (threadIdx.x == 0) tl_end(tl);
 }
 
 // Gather cached K/V rows into canonical [npos][Hkv][hd] order (debug read-back).

@@ -66,8 +66,12 @@ attn_replay_kernel(const bf16 *__restrict__ Q, const bf16 *__restrict__ Kpool, c
     const int t = t0 + lane;
     const bf16 *kr = nullptr, *vr = nullptr;
     if (t < nvis) {
-      const size_t off = kv_row_offset(g, seq, t, kvh);
-      kr = Kpool + off; vr = Vpool + off;
+      // a caller-provided table may hold anything: a key on a page outside the pool is skipped
+      const int page = g.page_table[(size_t)seq * g.pages_per_seq + t / g.page_size];
+      if (g.n_pages == 0 || (unsigned)page < (unsigned)g.n_pages) {
+        const size_t off = (((size_t)page * g.n_kv_heads + kvh) * g.page_size + (t % g.page_size)) * (size_t)g.head_dim;
+        kr = Kpool + off; vr = Vpool + off;
+      }
     } else if (t < total) {
       const size_t off = ((size_t)(loc0 + t - nvis) * g.n_kv_heads + kvh) * HD;
       kr = Kloc + off; vr = Vloc + off;
@@ -90,7 +94,9 @@ attn_replay_kernel(const bf16 *__restrict__ Q, const bf16 *__restrict__ Kpool, c
       sc = a;
     }
     const float nmx = fmaxf(mx, warp_max(sc));
-    const float corr = __expf(mx - nmx);           // mx = -inf on the first chunk gives 0
+    // mx = -inf before the first visible key gives 0; a chunk without any visible key while
+    // nothing has been seen yet (nmx = -inf) must leave the empty sums alone, not make them NaN
+    const float corr = nmx == -INFINITY ? 1.f : __expf(mx - nmx);
     const float p = kr ? __expf(sc - nmx) : 0.f;
     den = den * corr + warp_sum(p);
 #pragma unroll
@@ -100,11 +106,12 @@ attn_replay_kernel(const bf16 *__restrict__ Q, const bf16 *__restrict__ Kpool, c
     for (int j = 0; j < 32 && t0 + j < total; ++j) {
       const float pj = __shfl_sync(0xffffffffu, p, j);
       const bf16 *vj = (const bf16 *)__shfl_sync(0xffffffffu, vaddr, j);
+      if (vj == nullptr) continue;                 // a skipped key (page outside the pool): weight 0, nothing to read; same for every lane
 #pragma unroll
       for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pj, __bfloat162float(vj[lane * DPL + i]), acc[i]);
     }
   }
   bf16 *o = O + ((size_t)r * Hq + h) * HD;
 #pragma unroll
-  for (int i = 0; i < DPL; ++i) o[lane * DPL + i] = __float2bfloat16(acc[i] / den);
+  for (int i = 0; i < DPL; ++i) o[lane * DPL + i] = __float2bfloat16(den > 0.f ? acc[i] / den : 0.f);   // no visible key: zeros
 }

@@ -21,7 +21,7 @@ std::string g_init_error;
 
 struct SeqState {
   int n = 0;            // committed KV length
-  int k = 0;            // draft block length chosen at prefill
+  int k = 0;            // draft block length of the sequence's last pass (entries its block holds)
   bool active = false;
   std::vector<int> pages;
 };
@@ -44,6 +44,10 @@ struct tidar_ctx {
   // arena carve-out (device)
   bf16 *kv = nullptr;
   RowMeta meta{};
+  int32_t *d_blk_len = nullptr;    // [max_batch]: drafts a sequence's block holds (the block length of its last pass)
+  float *d_run_max = nullptr, *d_run_sum = nullptr, *d_tgt_logit = nullptr, *d_logprob = nullptr;   // likelihood scoring, per row
+  int32_t *d_target = nullptr;
+  std::vector<CUtensorMap> tm_lm_chunks;   // the LM head in vocabulary chunks of lm_chunk rows (scoring)
   int32_t *d_seq_len = nullptr, *d_block = nullptr, *d_page_table = nullptr, *d_step_seqs = nullptr, *d_forced = nullptr,
           *d_step_n = nullptr, *d_step_L = nullptr, *d_out = nullptr, *d_prompt = nullptr, *d_arg_idx = nullptr;
   float *X = nullptr, *partials = nullptr, *rope_cos = nullptr, *rope_sin = nullptr, *d_arg_val = nullptr,
@@ -58,7 +62,7 @@ struct tidar_ctx {
   int64_t launches = 0;
   // last pass
   int last_rows = 0, last_first_pos = 0;
-  std::vector<int> pending_seqs; std::vector<int> pending_forced; bool pending = false;
+  std::vector<int> pending_seqs; std::vector<int> pending_forced; bool pending = false; int pending_k = 0;
   // tensor-core path
   gemm_tc::EncodeTiledFn encode = nullptr;
   std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
@@ -69,12 +73,18 @@ struct tidar_ctx {
   float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
   // the launches of one decode step as an executable graph, valid for one (k, n_seqs, attention split)
-  struct StepGraph { int k = 0, n_seqs = 0, splits = 0; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
+  struct StepGraph { int k = 0, n_seqs = 0, splits = 0; bool ar = false, timeline = false; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
   bool graphs_ok = true;
   bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
   float *cand_val = nullptr;
   int32_t *h_status = nullptr;
+  // in-kernel timeline (diagnostics): two words per launch of the last recorded step
+  static constexpr int TL_MAX = 2048;
+  unsigned long long *d_tl = nullptr;
+  bool timeline = false; int tl_n = 0; std::vector<int> tl_cls;
+  bool count_tiles = false;        // the attention kernel adds the key tiles it visits to d_tl[2 * TL_MAX]
+  float tl_class_ms[TIDAR_TC_COUNT] = {}; float tl_span_ms = 0.f, tl_busy_ms = 0.f;
   // timing
   bool timing = false; std::vector<TimedLaunch> timed; float class_ms[TIDAR_TC_COUNT] = {};
   int cur_class = 0;
@@ -113,13 +123,15 @@ int validate(const tidar_config &c, std::string &why) {
   auto bad = [&](const char *m) { why = m; return TIDAR_EINVAL; };
   if (c.n_layers < 1 || c.d_model < 64 || c.vocab < 2 || c.d_ffn < 64) return bad("n_layers, d_model, d_ffn, vocab must be positive");
   if (c.head_dim != 64 && c.head_dim != 128) return bad("head_dim must be 64 or 128");
-  if (c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads) return bad("n_q_heads must be a multiple of n_kv_heads");
+  if (c.n_kv_heads < 1 || c.n_q_heads < 1 || c.n_q_heads % c.n_kv_heads) return bad("n_q_heads must be a positive multiple of n_kv_heads");
+  if (c.n_q_heads / c.n_kv_heads > 128) return bad("at most 128 query heads per KV head (one 128-row attention tile)");
+  if (c.d_model > 12288) return bad("d_model above 12288 is not supported (row buffer of the norm kernel)");
   if (c.d_model % 64 || c.d_ffn % 64) return bad("d_model and d_ffn must be multiples of 64");
   if (c.page_size != 64) return bad("page_size must be 64");
   if (c.k_max < 1 || c.k_max > 32) return bad("k_max must be in [1, 32]");
   if (c.max_batch < 1 || c.max_seq_len < 2 * c.k_max + 1) return bad("max_batch >= 1 and max_seq_len > 2*k_max required");
   if (c.mask_token_id < 0 || c.mask_token_id >= c.vocab) return bad("mask_token_id out of range");
-  if (c.beta != 1.0f) return bad("only beta = 1 is implemented");
+  if (!(c.beta >= 0.0f && c.beta <= 1.0f)) return bad("beta must be in [0, 1]");
   if (c.temperature != 0.0f) return bad("only greedy decoding (temperature 0) is implemented");
   if (c.impl != 0 && c.impl != 1) return bad("impl must be 0 (tensor-core kernels) or 1 (replay kernels)");
   if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return bad("rms_eps > 0 and rope_theta > 1 required");
@@ -129,7 +141,8 @@ int validate(const tidar_config &c, std::string &why) {
 void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   const tidar_config &c = x.cfg;
   x.T_max = c.k_max * (c.k_max + 1);
-  x.R_cap = (int)align_up((size_t)std::max(c.max_batch * x.T_max, 256), 16);
+  // rows of a pass: the step's slots, plus one mixed row per verified position when beta < 1
+  x.R_cap = (int)align_up((size_t)std::max(c.max_batch * (x.T_max + (c.beta < 1.0f ? c.k_max : 0)), 256), 16);
   x.pages_per_seq = (c.max_seq_len + c.page_size - 1) / c.page_size;
   x.n_pages = x.pages_per_seq * c.max_batch;
   x.n_qkv = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
@@ -146,6 +159,9 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.meta.nvis = cv.take<int32_t>(R); x.meta.loc0 = cv.take<int32_t>(R); x.meta.nloc = cv.take<int32_t>(R);
   x.meta.cache_pos = cv.take<int32_t>(R); x.meta.local_idx = cv.take<int32_t>(R);
   x.d_seq_len = cv.take<int32_t>(c.max_batch);
+  x.d_blk_len = cv.take<int32_t>(c.max_batch);
+  x.d_run_max = cv.take<float>(R); x.d_run_sum = cv.take<float>(R); x.d_tgt_logit = cv.take<float>(R); x.d_logprob = cv.take<float>(R);
+  x.d_target = cv.take<int32_t>(R);
   x.d_block = cv.take<int32_t>((size_t)c.max_batch * c.k_max);
   x.d_page_table = cv.take<int32_t>((size_t)c.max_batch * x.pages_per_seq);
   x.d_step_seqs = cv.take<int32_t>(c.max_batch); x.d_forced = cv.take<int32_t>(c.max_batch);
@@ -154,6 +170,7 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.d_prompt = cv.take<int32_t>(c.max_seq_len);
   x.d_arg_idx = cv.take<int32_t>(R); x.d_arg_val = cv.take<float>(R);
   x.d_status = cv.take<int32_t>(64);
+  x.d_tl = cv.take<unsigned long long>(2 * tidar_ctx::TL_MAX + 8);   // timeline slots, then diagnostic counters
   if (c.impl == 0) {
     x.attn_part_O = cv.take<float>((size_t)attn_tc::MAX_SPLITS * R * c.n_q_heads * c.head_dim);
     x.attn_part_ml = cv.take<float>((size_t)attn_tc::MAX_SPLITS * R * c.n_q_heads * 2);
@@ -213,10 +230,11 @@ inline void launch_after(void (*kernel)(KP...), dim3 grid, dim3 block, size_t sm
 
 // ---- launch bookkeeping -----------------------------------------------------
 struct Launch {
-  tidar_ctx *c; int cls; cudaEvent_t a = nullptr, b = nullptr;
+  tidar_ctx *c; int cls; cudaEvent_t a = nullptr, b = nullptr; TlSlot tl{nullptr};
   Launch(tidar_ctx *c_, int cls_) : c(c_), cls(cls_) {
     c->launches++;
     if (c->timing) { cudaEventCreate(&a); cudaEventCreate(&b); cudaEventRecord(a, c->stream); }
+    if (c->timeline && c->tl_n < tidar_ctx::TL_MAX) { tl.t = c->d_tl + 2 * c->tl_n; c->tl_n++; c->tl_cls.push_back(cls); }
   }
   ~Launch() {
     if (c->timing) { cudaEventRecord(b, c->stream); c->timed.push_back({cls, a, b}); }
@@ -233,8 +251,28 @@ void collect_timing(tidar_ctx *c) {
   c->timed.clear();
 }
 
+// Per class, the sum over the last step's launches of (latest CTA end - earliest CTA start);
+// busy = the sum over all launches, span = first start to last end.
+void collect_timeline(tidar_ctx *c) {
+  std::vector<unsigned long long> h(2 * (size_t)c->tl_n);
+  for (int i = 0; i < TIDAR_TC_COUNT; ++i) c->tl_class_ms[i] = 0.f;
+  c->tl_span_ms = c->tl_busy_ms = 0.f;
+  if (c->tl_n == 0) return;
+  if (cudaMemcpy(h.data(), c->d_tl, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return; }
+  unsigned long long first = ~0ull, last = 0;
+  for (int i = 0; i < c->tl_n; ++i) {
+    if (h[2 * i] == 0 || h[2 * i + 1] == 0) continue;          // a launch that stamped nothing
+    const unsigned long long t0 = ~h[2 * i], t1 = h[2 * i + 1];
+    if (t1 < t0) continue;
+    const float ms = (float)((double)(t1 - t0) * 1e-6);
+    c->tl_class_ms[c->tl_cls[i]] += ms; c->tl_busy_ms += ms;
+    first = std::min(first, t0); last = std::max(last, t1);
+  }
+  if (last > first) c->tl_span_ms = (float)((double)(last - first) * 1e-6);
+}
+
 KvGeom geom(const tidar_ctx *c) {
-  return KvGeom{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, c->pages_per_seq, c->d_page_table};
+  return KvGeom{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, c->pages_per_seq, c->d_page_table, 0};
 }
 
 // ---- projections --------------------------------------------------------------
@@ -310,19 +348,19 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   const int grid = std::min(items, c->n_sms);
   const size_t smem = gemm_tc::smem_bytes(a);
   Launch l(c, cls);
-  if (mode == gemm_tc::MODE_SLAB) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
-  else if (mode == gemm_tc::MODE_SWIGLU) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
-  else launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a);
+  if (mode == gemm_tc::MODE_SLAB) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
+  else if (mode == gemm_tc::MODE_SWIGLU) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
+  else launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
   if (rem_tiles) {
     const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
     const size_t n = (size_t)R * nf;
-    c->launches++;
+    Launch lf(c, cls);
     if (c->slab_bf16)
       launch_after(swiglu_slab_kernel<bf16>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const bf16 *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
-                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
+                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H, lf.tl);
     else
       launch_after(swiglu_slab_kernel<float>, (unsigned)((n / 2 + 255) / 256), 256, 0, c->stream, (const float *)c->partials, a.S, (size_t)a.slab_stride, R, a.ldo, nf,
-                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H);
+                                                                           a.tile_b0 * gemm_tc::TILE_N / 2, a.ldh, c->H, lf.tl);
   }
   if (S_out) *S_out = a.S;
   if (stride_out) *stride_out = (size_t)R * N;
@@ -401,21 +439,22 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   a.page_base_k = m.page_base_k; a.page_base_v = m.page_base_v;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)cf.head_dim);
   a.O = O; a.part_O = c->attn_part_O; a.part_ml = c->attn_part_ml; a.status = c->d_status;
+  a.tile_count = c->count_tiles ? c->d_tl + 2 * tidar_ctx::TL_MAX : nullptr;
   const int grid = units * a.splits;
   {
     Launch l(c, TIDAR_TC_ATTN);
     if (cf.head_dim == 128)
-      launch_pdl(attn_tc::attn_tc_kernel<128>, grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      launch_pdl(attn_tc::attn_tc_kernel<128>, grid, attn_tc::THREADS, attn_tc::Smem<128>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a, l.tl);
     else
-      launch_pdl(attn_tc::attn_tc_kernel<64>, grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a);
+      launch_pdl(attn_tc::attn_tc_kernel<64>, grid, attn_tc::THREADS, attn_tc::Smem<64>::TOTAL, c->stream, *m.q, *m.k, *m.v, *m.kloc, *m.vloc, a, l.tl);
   }
   if (a.splits > 1) {
     Launch l(c, TIDAR_TC_ATTN);
     const size_t threads = (size_t)R * cf.n_q_heads * (cf.head_dim / 4);
     if (cf.head_dim == 128)
-      launch_after(attn_tc::attn_combine_kernel<128>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<128>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O, l.tl);
     else
-      launch_after(attn_tc::attn_combine_kernel<64>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O);
+      launch_after(attn_tc::attn_combine_kernel<64>, (unsigned)((threads + 255) / 256), 256, 0, c->stream, c->attn_part_O, c->attn_part_ml, a.splits, R, cf.n_q_heads, O, l.tl);
   }
 }
 
@@ -435,21 +474,24 @@ void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t strid
   Launch l(c, TIDAR_TC_NORM);
   const int d = c->cfg.d_model;
   if (c->cfg.impl == 0 && c->slab_bf16)
-    launch_after(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+    launch_after(rmsnorm_reduce_kernel<512, bf16>, R, 512, d * sizeof(float), c->stream, c->X, (const bf16 *)partials, S, stride, gain, c->cfg.rms_eps, d, c->A, l.tl);
   else
-    launch_after(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A);
+    launch_after(rmsnorm_reduce_kernel<512, float>, R, 512, d * sizeof(float), c->stream, c->X, partials, S, stride, gain, c->cfg.rms_eps, d, c->A, l.tl);
 }
 
 // The transformer stack over R assembled rows (metadata and X already filled).
 // with_head: run final norm + LM head + per-row argmax.
-int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int key_tiles_hint) {
+// Extra LM-head input rows that mix two final-normed rows each (beta < 1; see mix_rows_kernel).
+struct MixRows { int n = 0, k = 1, a0 = 0, a_seq = 0, a_j = 0, b0 = 0, b_seq = 0, b_j = 0; };
+
+int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int key_tiles_hint, const MixRows &mix = MixRows()) {
   const tidar_config &cf = c->cfg;
   const int d = cf.d_model, hd = cf.head_dim, Hq = cf.n_q_heads, Hkv = cf.n_kv_heads;
   const KvGeom g = geom(c);
   {
     Launch l(c, TIDAR_TC_ROPE);
     const int n = R * (hd / 2);
-    launch_after(rope_table_kernel, (n + 255) / 256, 256, 0, c->stream, c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin);
+    launch_after(rope_table_kernel, (n + 255) / 256, 256, 0, c->stream, c->meta.pos, R, hd / 2, (double)cf.rope_theta, c->rope_cos, c->rope_sin, l.tl);
   }
   int S = 0; size_t stride = 0;          // pending partials of the previous down projection
   const bool tc = cf.impl == 0;
@@ -467,10 +509,10 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
       const int rope_chunks = ((Hq + 2 * Hkv) * (hd / 8) + 255) / 256;
 if (tc && c->slab_bf16)
         launch_after(rope_kv_kernel<bf16>, dim3(R, rope_chunks), 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
-                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, ll.tl);
       else
         launch_after(rope_kv_kernel<float>, dim3(R, rope_chunks), 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
-                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc);
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, ll.tl);
     }
     if (tc) {
       AttnMaps am{&c->tm_q, &c->tm_kv, &c->tm_kv, &c->tm_kloc, &c->tm_vloc, (2 * l) * c->n_pages, (2 * l + 1) * c->n_pages};
@@ -494,12 +536,17 @@ if (tc && c->slab_bf16)
   if (c->dbg_hidden)
     CUDA_TRY(c, cudaMemcpyAsync(c->dbg_hidden + (size_t)cf.n_layers * c->R_cap * d, c->X, (size_t)R * d * sizeof(float),
                                 cudaMemcpyDeviceToDevice, c->stream));
+  if (with_head && mix.n > 0) {            // rows R .. R + mix.n - 1 of the LM head's input
+    Launch lm(c, TIDAR_TC_NORM);
+    launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, R, lm.tl);
+    R += mix.n;
+  }
   if (with_head && tc) {
     const int G = c->n_sms * 4;          // upper bound of (CTAs of the LM-head kernel) x 4 lane quadrants
     CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
     if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    launch_after(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx);
+    launch_after(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx, ll.tl);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
@@ -534,6 +581,11 @@ int init_tensor_core_path(tidar_ctx *c) {
   };
   c->tm_wqkv.resize(cf.n_layers); c->tm_wo.resize(cf.n_layers); c->tm_wgu.resize(cf.n_layers); c->tm_wdown.resize(cf.n_layers);
   bool ok = enc(&c->tm_lm, c->lm_head, cf.vocab, d);
+  c->tm_lm_chunks.resize((cf.vocab + c->lm_chunk - 1) / c->lm_chunk);
+  for (size_t ci = 0; ci < c->tm_lm_chunks.size() && ok; ++ci) {
+    const int v0 = (int)ci * c->lm_chunk;
+    ok = enc(&c->tm_lm_chunks[ci], c->lm_head + (size_t)v0 * d, std::min(c->lm_chunk, cf.vocab - v0), d);
+  }
   for (int l = 0; l < cf.n_layers && ok; ++l)
     ok = enc(&c->tm_wqkv[l], c->wqkv[l], c->n_qkv, d) && enc(&c->tm_wo[l], c->wo[l], d, qo) &&
          enc(&c->tm_wgu[l], c->wgu[l], 2 * cf.d_ffn, d) && enc(&c->tm_wdown[l], c->wdown[l], d, cf.d_ffn);
@@ -572,6 +624,13 @@ int check_device_status(tidar_ctx *c) {
   return TIDAR_OK;
 }
 
+// Returns a sequence slot's pages to the pool and marks it as not prefilled.
+void release_sequence(tidar_ctx *c, int seq) {
+  SeqState &s = c->seqs[seq];
+  for (int p : s.pages) c->free_pages.push_back(p);
+  s.pages.clear(); s.active = false; s.n = 0;
+}
+
 int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
   SeqState &s = c->seqs[seq];
   const int need = (upto_positions + c->cfg.page_size - 1) / c->cfg.page_size;
@@ -590,26 +649,35 @@ int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
 }
 
 // Enqueues every operation of one decode step for the sequences staged in h_stage.
-int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint) {
+// k: block length of this step; ar: plain autoregressive step (the causal section alone).
+int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar) {
   const tidar_config &cf = c->cfg;
-  const int T = k * (k + 1), R = n_seqs * T;
+  const int n_blocks = ar ? 0 : k;
+  const int T = k * (n_blocks + 1), R = n_seqs * T;
+  if (c->timeline) {
+    c->tl_n = 0; c->tl_cls.clear();
+    CUDA_TRY(c, cudaMemsetAsync(c->d_tl, 0, 2 * tidar_ctx::TL_MAX * sizeof(unsigned long long), c->stream));
+  }
   CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
-    launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, k, cf.k_max, cf.mask_token_id,
-               c->d_step_n, c->embed, cf.d_model, c->X);
+    launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, c->d_blk_len, k, n_blocks, cf.k_max,
+               cf.mask_token_id, c->d_step_n, c->embed, cf.d_model, c->X, l.tl);
   }
-  if (int rc = forward_rows(c, R, true, T, key_tiles_hint)) return rc;
+  // beta < 1: the verified prediction of causal slot j mixes its row with the first slot of block j
+  MixRows mix;
+  if (cf.beta < 1.0f && !ar) { mix.n = n_seqs * k; mix.k = k; mix.a0 = 0; mix.a_seq = T; mix.a_j = 1; mix.b0 = k; mix.b_seq = T; mix.b_j = k; }
+  if (int rc = forward_rows(c, R, true, T, key_tiles_hint, mix)) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    launch_after(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, c->d_step_seqs, c->d_forced, k, cf.k_max, c->d_block,
-               c->d_step_L, c->d_out);
+    launch_after(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, mix.n ? c->d_arg_idx + R : (const int32_t *)nullptr, c->d_step_seqs,
+               c->d_forced, k, n_blocks, cf.k_max, c->d_block, c->d_blk_len, c->d_step_L, c->d_out, l.tl);
   }
   {
     Launch l(c, TIDAR_TC_VERIFY);
     launch_after(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
-               (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride);
+               (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride, l.tl);
   }
   CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
@@ -617,28 +685,32 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint) {
   return TIDAR_OK;
 }
 
-int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced) {
+// k_step: block length of this step (0 = the one the sequences' last pass left, which must then be
+// the same for all of them); ar: plain autoregressive step (k_step is 1).
+int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced, int k_step = 0, bool ar = false) {
   const tidar_config &cf = c->cfg;
   if (!seqs || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
   if (c->pending) return fail(c, TIDAR_EINVAL, "a step is already in flight; call tidar_step_wait first");
-  int k = 0;
+  if (k_step < 0 || k_step > cf.k_max) return fail(c, TIDAR_EINVAL, "block length %d outside [1, k_max = %d]", k_step, cf.k_max);
+  int k = ar ? 1 : k_step;
   for (int i = 0; i < n_seqs; ++i) {
     const int q = seqs[i];
     if (q < 0 || q >= cf.max_batch || !c->seqs[q].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", q);
     for (int j = 0; j < i; ++j) if (seqs[j] == q) return fail(c, TIDAR_EINVAL, "sequence %d listed twice", q);
-    if (i == 0) k = c->seqs[q].k;
-    else if (c->seqs[q].k != k) return fail(c, TIDAR_EINVAL, "all sequences of a step must share one draft length k");
+    if (k == 0) k = c->seqs[q].k;
+    else if (k_step == 0 && !ar && c->seqs[q].k != k)
+      return fail(c, TIDAR_EINVAL, "the listed sequences hold blocks of different lengths; name the step's block length (tidar_step_k)");
     const int f = forced ? forced[i] : 0;
     if (f < 0 || f > k) return fail(c, TIDAR_EINVAL, "forced acceptance %d outside [0, %d]", f, k);
     if (need_forced && f == 0) return fail(c, TIDAR_EINVAL, "tidar_step_async needs a forced acceptance length per sequence");
-    if (c->seqs[q].n + 2 * k > cf.max_seq_len)
-      return fail(c, TIDAR_ECAPACITY, "sequence %d: n + 2k = %d exceeds max_seq_len %d", q, c->seqs[q].n + 2 * k, cf.max_seq_len);
+    if (c->seqs[q].n + (ar ? 1 : 2 * k) > cf.max_seq_len)
+      return fail(c, TIDAR_ECAPACITY, "sequence %d: n + %s = %d exceeds max_seq_len %d", q, ar ? "1" : "2k", c->seqs[q].n + (ar ? 1 : 2 * k), cf.max_seq_len);
   }
   for (int i = 0; i < n_seqs; ++i) {
     int rc = ensure_pages(c, seqs[i], c->seqs[seqs[i]].n + k);
     if (rc) return rc;
   }
-  const int T = k * (k + 1), R = n_seqs * T;
+  const int T = ar ? 1 : k * (k + 1), R = n_seqs * T;
   for (int i = 0; i < n_seqs; ++i) { c->h_stage[i] = seqs[i]; c->h_stage[cf.max_batch + i] = forced ? forced[i] : 0; }
   int min_n = 1 << 30;
   for (int i = 0; i < n_seqs; ++i) min_n = std::min(min_n, c->seqs[seqs[i]].n);
@@ -652,14 +724,14 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
     const int G = cf.n_q_heads / cf.n_kv_heads, spt = 128 / G;
     const int splits = attn_key_splits(c, n_seqs * ((T + spt - 1) / spt) * cf.n_kv_heads, hint);
     tidar_ctx::StepGraph &sg = c->sg;
-    if (!sg.exec || sg.k != k || sg.n_seqs != n_seqs || sg.splits != splits) {
+    if (!sg.exec || sg.k != k || sg.ar != ar || sg.n_seqs != n_seqs || sg.splits != splits || sg.timeline != c->timeline) {
       if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
       const int64_t l0 = c->launches;
       cudaGraph_t graph = nullptr;
       int rc = TIDAR_OK;
       cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
       if (e == cudaSuccess) {
-        rc = record_step(c, n_seqs, k, hint);
+        rc = record_step(c, n_seqs, k, hint, ar);
         e = cudaStreamEndCapture(c->stream, &graph);
       }
       if (e == cudaSuccess && rc == TIDAR_OK && graph) e = cudaGraphInstantiate(&sg.exec, graph, 0);
@@ -668,7 +740,7 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
         cudaGetLastError();                         // capture is not available here: plain launches from now on
         sg.exec = nullptr; c->graphs_ok = false;
       } else {
-        sg.k = k; sg.n_seqs = n_seqs; sg.splits = splits; sg.launches = c->launches - l0;
+        sg.k = k; sg.ar = ar; sg.n_seqs = n_seqs; sg.splits = splits; sg.timeline = c->timeline; sg.launches = c->launches - l0;
       }
       c->launches = l0;
     }
@@ -679,10 +751,11 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
     }
   }
   if (!launched)
-    if (int rc = record_step(c, n_seqs, k, hint)) return rc;
+    if (int rc = record_step(c, n_seqs, k, hint, ar)) return rc;
+  c->pending_k = k;
   c->pending_seqs.assign(seqs, seqs + n_seqs);
   c->pending = true;
-  c->last_rows = R; c->last_first_pos = -1;
+  c->last_rows = R + ((cf.beta < 1.0f && !ar) ? n_seqs * k : 0); c->last_first_pos = -1;      // the mixed rows follow the slots
   // the host tracks lengths without reading the device when L is forced
   return TIDAR_OK;
 }
@@ -692,12 +765,21 @@ int finish_step(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
   c->pending = false;
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   if (c->timing) collect_timing(c);
-  if (c->h_status[0]) { c->h_status[0] = 0; cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
-    return fail(c, TIDAR_EDEVICE_TIMEOUT, "a bounded device-side wait gave up during the step; its results are invalid"); }
+  if (c->timeline) collect_timeline(c);
+  if (c->h_status[0]) {
+    // The step's kernels have already rewritten the device-side lengths and blocks of the listed
+    // sequences from invalid results: their state is lost.  Release them; a new first pass is needed.
+    const int st = c->h_status[0];
+    c->h_status[0] = 0; cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
+    for (int q : c->pending_seqs) release_sequence(c, q);
+    return fail(c, TIDAR_EDEVICE_TIMEOUT, "a bounded device-side wait gave up during the step (status %d); its results are invalid and the "
+                                          "listed sequences were released (prefill them again)", st);
+  }
   const int km = c->cfg.k_max;
   for (size_t i = 0; i < c->pending_seqs.size(); ++i) {
     const int L = c->h_pinned[i * (km + 1)];
     c->seqs[c->pending_seqs[i]].n += L;
+    c->seqs[c->pending_seqs[i]].k = c->pending_k;        // the block the step left has this many entries
     if (out_n) out_n[i] = L;
     if (out_tokens) for (int j = 0; j < km; ++j) out_tokens[i * km + j] = j < L ? c->h_pinned[i * (km + 1) + 1 + j] : -1;
   }
@@ -778,12 +860,12 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
   for (int i = 0; i < n_prompt; ++i)
     if (prompt[i] < 0 || prompt[i] >= cf.vocab) return fail(c, TIDAR_EINVAL, "prompt id %d at %d out of range", prompt[i], i);
   SeqState &s = c->seqs[seq];
-  for (int p : s.pages) c->free_pages.push_back(p);
-  s.pages.clear(); s.active = false; s.n = 0; s.k = k;
+  release_sequence(c, seq);
+  s.k = k;
   if (int rc = ensure_pages(c, seq, n_prompt + k)) return rc;
   CUDA_TRY(c, cudaMemcpyAsync(c->d_prompt, prompt, (size_t)n_prompt * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   const int total = n_prompt + k;
-  const int last_rows = std::min(total, c->R_cap);
+  const int last_rows = std::min(total, c->R_cap - (cf.beta < 1.0f ? 1 : 0));     // the last chunk may carry one mixed row
   int row0 = 0;
   while (row0 < total) {
     const bool last = row0 >= total - last_rows;
@@ -793,11 +875,15 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
       assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
                                                            cf.d_model, c->X);
     }
-    if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64)) return rc;
+    // beta < 1: the settled first token mixes the last prompt row with the first mask row
+    MixRows mix;
+    const int rlp = n_prompt - 1 - row0;               // the last prompt row inside this chunk
+    if (last && cf.beta < 1.0f) { mix.n = 1; mix.k = 1; mix.a0 = rlp; mix.b0 = rlp + 1; }
+    if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64, mix)) return rc;
     if (last) {
       Launch l(c, TIDAR_TC_VERIFY);
-      prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, n_prompt - 1 - row0, k, cf.k_max, seq, n_prompt, c->d_block,
-                                                     c->d_seq_len, c->d_out);
+      prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, rlp, mix.n ? rows : rlp, k, cf.k_max, seq, n_prompt, c->d_block,
+                                                     c->d_blk_len, c->d_seq_len, c->d_out);
       c->last_rows = rows; c->last_first_pos = row0;
     }
     row0 += rows;
@@ -806,7 +892,7 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   CUDA_TRY(c, cudaGetLastError());
   if (c->timing) collect_timing(c);
-  if (int rc = check_device_status(c)) return rc;
+  if (int rc = check_device_status(c)) { release_sequence(c, seq); return rc; }
   s.n = n_prompt; s.active = true;
   if (out_first) *out_first = c->h_pinned[0];
   return TIDAR_OK;
@@ -827,6 +913,75 @@ int tidar_step_async(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, const in
 int tidar_step_wait(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
   if (!c) return TIDAR_EINVAL;
   return finish_step(c, out_tokens, out_n);
+}
+
+int tidar_step_k(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t k, const int32_t *forced, int32_t *out_tokens, int32_t *out_n) {
+  if (!c) return TIDAR_EINVAL;
+  if (k < 1) return fail(c, TIDAR_EINVAL, "block length must be at least 1");
+  if (int rc = enqueue_step(c, seqs, n_seqs, forced, false, k, false)) return rc;
+  return finish_step(c, out_tokens, out_n);
+}
+
+int tidar_ar_step(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t *out_tokens) {
+  if (!c) return TIDAR_EINVAL;
+  if (int rc = enqueue_step(c, seqs, n_seqs, nullptr, false, 1, true)) return rc;
+  std::vector<int32_t> toks((size_t)std::max(n_seqs, 1) * c->cfg.k_max), ls(std::max(n_seqs, 1));
+  if (int rc = finish_step(c, toks.data(), ls.data())) return rc;
+  if (out_tokens) for (int i = 0; i < n_seqs; ++i) out_tokens[i] = toks[(size_t)i * c->cfg.k_max];
+  return TIDAR_OK;
+}
+
+int tidar_ridge_k(const tidar_ctx *c, int32_t n_seqs, int32_t row_budget) {
+  if (!c || n_seqs < 1) return TIDAR_EINVAL;
+  if (row_budget <= 0) row_budget = 288;       // one row block of the projections: where the 8B-class step turns tensor-bound
+  int k = 1;
+  while (k < c->cfg.k_max && (long long)n_seqs * (k + 1) * (k + 2) <= row_budget) ++k;
+  return k;
+}
+
+int tidar_score(tidar_ctx *c, int32_t seq, const int32_t *ids, int32_t n, float *logprobs) {
+  if (!c) return TIDAR_EINVAL;
+  const tidar_config &cf = c->cfg;
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (seq < 0 || seq >= cf.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
+  if (!ids || !logprobs || n < 2) return fail(c, TIDAR_EINVAL, "tidar_score needs at least two token ids");
+  if (n > cf.max_seq_len) return fail(c, TIDAR_ECAPACITY, "%d tokens exceed max_seq_len %d", n, cf.max_seq_len);
+  for (int i = 0; i < n; ++i)
+    if (ids[i] < 0 || ids[i] >= cf.vocab) return fail(c, TIDAR_EINVAL, "token id %d at %d out of range", ids[i], i);
+  release_sequence(c, seq);
+  c->seqs[seq].k = 1;
+  if (int rc = ensure_pages(c, seq, n)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_prompt, ids, (size_t)n * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  const int d = cf.d_model;
+  for (int row0 = 0; row0 < n - 1; row0 += c->R_cap) {
+    const int rows = std::min(c->R_cap, n - 1 - row0);          // the last token predicts nothing that is scored
+    {
+      Launch l(c, TIDAR_TC_EMBED);
+      assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n, 0, cf.mask_token_id, c->d_prompt, c->embed, d, c->X);
+    }
+    if (int rc = forward_rows(c, rows, false, rows, (row0 + rows / 2 + 63) / 64)) return rc;      // ends with the final norm in c->A
+    for (int v0 = 0, ci = 0; v0 < cf.vocab; v0 += c->lm_chunk, ++ci) {
+      const int nc = std::min(c->lm_chunk, cf.vocab - v0);
+      int S = 1; size_t stride = 0;
+      if (cf.impl == 0) {
+        if (int rc = gemm_tc_launch(c, gemm_tc::MODE_SLAB, c->A, c->R_cap, c->tm_lm_chunks[ci], rows, nc, d, TIDAR_TC_LMHEAD, &S, &stride, c->partials, 1)) return rc;
+      } else {
+        if (int rc = gemm_partials(c, c->A, c->R_cap, c->lm_head + (size_t)v0 * d, nullptr, rows, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD)) return rc;
+      }
+      Launch ll(c, TIDAR_TC_LMHEAD);
+      score_chunk_kernel<<<rows, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_prompt + row0 + 1, c->d_run_max, c->d_run_sum, c->d_tgt_logit);
+    }
+    {
+      Launch ll(c, TIDAR_TC_LMHEAD);
+      score_finish_kernel<<<(rows + 127) / 128, 128, 0, c->stream>>>(c->d_run_max, c->d_run_sum, c->d_tgt_logit, rows, c->d_logprob);
+    }
+    CUDA_TRY(c, cudaMemcpyAsync(logprobs + row0, c->d_logprob, (size_t)rows * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  }
+  CUDA_TRY(c, cudaGetLastError());
+  if (c->timing) collect_timing(c);
+  release_sequence(c, seq);                         // the slot was scratch for this call
+  return check_device_status(c);
 }
 
 int tidar_free(tidar_ctx *c) {
@@ -852,6 +1007,7 @@ int tidar_debug_set_block(tidar_ctx *c, int32_t seq, const int32_t *block) {
   if (!c || !block) return TIDAR_EINVAL;
   if (seq < 0 || seq >= c->cfg.max_batch || !c->seqs[seq].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", seq);
   CUDA_TRY(c, cudaMemcpyAsync(c->d_block + (size_t)seq * c->cfg.k_max, block, c->seqs[seq].k * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_blk_len + seq, &c->seqs[seq].k, sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return TIDAR_OK;
 }
@@ -923,6 +1079,44 @@ int tidar_debug_get_kv(tidar_ctx *c, int32_t seq, int32_t layer, int32_t pos0, i
   return TIDAR_OK;
 }
 
+int tidar_debug_force_status(tidar_ctx *c, int32_t value) {
+  if (!c) return TIDAR_EINVAL;
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_status, &value, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return TIDAR_OK;
+}
+
+int tidar_debug_count_attention_tiles(tidar_ctx *c, int32_t on, uint64_t *visited) {
+  if (!c) return TIDAR_EINVAL;
+  if (c->cfg.impl != 0) return fail(c, TIDAR_EINVAL, "the tile counter exists for the tensor-core attention kernel only");
+  unsigned long long *ctr = c->d_tl + 2 * tidar_ctx::TL_MAX;
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (visited) {
+    unsigned long long v = 0;
+    CUDA_TRY(c, cudaMemcpy(&v, ctr, sizeof v, cudaMemcpyDeviceToHost));
+    *visited = v;
+  }
+  CUDA_TRY(c, cudaMemset(ctr, 0, sizeof(unsigned long long)));
+  if ((on != 0) != c->count_tiles && c->sg.exec) { cudaGraphExecDestroy(c->sg.exec); c->sg.exec = nullptr; }   // the flag is baked into the graph
+  c->count_tiles = on != 0;
+  return TIDAR_OK;
+}
+
+int tidar_debug_set_timeline(tidar_ctx *c, int32_t on) {
+  if (!c) return TIDAR_EINVAL;
+  if (c->cfg.impl != 0) return fail(c, TIDAR_EINVAL, "the in-kernel timeline exists for the tensor-core kernels only");
+  c->timeline = on != 0;
+  return TIDAR_OK;
+}
+
+int tidar_debug_get_timeline(tidar_ctx *c, float *class_ms, float *busy_ms, float *span_ms) {
+  if (!c || !class_ms) return TIDAR_EINVAL;
+  for (int i = 0; i < TIDAR_TC_COUNT; ++i) class_ms[i] = c->tl_class_ms[i];
+  if (busy_ms) *busy_ms = c->tl_busy_ms;
+  if (span_ms) *span_ms = c->tl_span_ms;
+  return TIDAR_OK;
+}
+
 int tidar_debug_set_timing(tidar_ctx *c, int32_t on) {
   if (!c) return TIDAR_EINVAL;
   c->timing = on != 0;
@@ -975,16 +1169,18 @@ int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void
   if (!q || !k_pages || !v_pages || !page_table || !seq_len || !k_local || !v_local || !out) return fail(c, TIDAR_EINVAL, "null argument");
   if (k < 1 || k > c->cfg.k_max || n_seqs < 1 || n_seqs * k * (k + 1) > c->R_cap) return fail(c, TIDAR_EINVAL, "n_seqs * k(k+1) exceeds the context's row capacity");
   if (n_pages < 1 || pages_per_seq < 1) return fail(c, TIDAR_EINVAL, "n_pages and pages_per_seq must be positive");
+  if ((long long)pages_per_seq * c->cfg.page_size < k) return fail(c, TIDAR_EINVAL, "the page table cannot back the k causal slots");
   if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)k_local | (uintptr_t)v_local | (uintptr_t)out) % 16 ||
+      ((uintptr_t)page_table | (uintptr_t)seq_len) % 4)
+    return fail(c, TIDAR_EINVAL, "tensors must be 16-byte aligned (page_table and seq_len 4-byte)");
   const int R = n_seqs * k * (k + 1);
   {
     Launch l(c, TIDAR_TC_EMBED);
-    attn_meta_kernel<<<(R + 127) / 128, 128, 0, c->stream>>>(c->meta, seq_len, k, R);
+    attn_meta_kernel<<<(R + 127) / 128, 128, 0, c->stream>>>(c->meta, seq_len, k, R, pages_per_seq * c->cfg.page_size - k);
   }
-  KvGeom g{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, pages_per_seq, page_table};
+  KvGeom g{c->cfg.n_kv_heads, c->cfg.head_dim, c->cfg.page_size, pages_per_seq, page_table, n_pages};
   if (c->cfg.impl == 0) {
-    if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)k_local | (uintptr_t)v_local | (uintptr_t)out) % 16)
-      return fail(c, TIDAR_EINVAL, "tensors must be 16-byte aligned");
     CUtensorMap tq, tk, tv, tkl, tvl;
     if (!encode_q_map(c, &tq, q, R) || !encode_pages_map(c, &tk, k_pages, n_pages) || !encode_pages_map(c, &tv, v_pages, n_pages) ||
         !encode_local_map(c, &tkl, k_local, (long long)n_seqs * k * k) || !encode_local_map(c, &tvl, v_local, (long long)n_seqs * k * k))
@@ -1026,7 +1222,7 @@ namespace {
 int32_t *g_static_ptr[TIDAR_STATIC_MAX_DEVICES] = {};
 }  // namespace
 
-extern "C" int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+extern "C" int tidar_attention_static(const void *q, const void *k_pages, const void *v_pages, int32_t n_pages, const int32_t *page_table,
                                       int32_t pages_per_seq, const int32_t *seq_len, const void *k_local, const void *v_local,
                                       void *out, int32_t n_seqs, int32_t k, int32_t n_q_heads, int32_t n_kv_heads,
                                       int32_t head_dim, void *cuda_stream) {
@@ -1035,7 +1231,13 @@ extern "C" int tidar_attention_static(const void *q, const void *k_pages, const 
   if (head_dim != 64 && head_dim != 128) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: head_dim must be 64 or 128");
   if (n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads)
     return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: n_q_heads must be a positive multiple of n_kv_heads");
-  if (k < 1 || k > 32 || n_seqs < 1 || pages_per_seq < 1) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: bad k, n_seqs or pages_per_seq");
+  if (k < 1 || k > 32 || n_seqs < 1 || pages_per_seq < 1 || n_pages < 1)
+    return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: bad k, n_seqs, n_pages or pages_per_seq");
+  if ((long long)pages_per_seq * 64 < k) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: the page table cannot back the k causal slots");
+  // the kernel reads K/V rows with 16-byte loads
+  if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)k_local | (uintptr_t)v_local | (uintptr_t)out) % 16 ||
+      ((uintptr_t)page_table | (uintptr_t)seq_len) % 4)
+    return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: tensors must be 16-byte aligned (page_table and seq_len 4-byte)");
   const long long rows = (long long)n_seqs * k * (k + 1);
   if (rows > TIDAR_STATIC_MAX_ROWS)
     return fail(nullptr, TIDAR_ECAPACITY, "tidar_attention_static: %lld rows exceed the built-in table of %d rows; use tidar_attention",
@@ -1043,7 +1245,9 @@ extern "C" int tidar_attention_static(const void *q, const void *k_pages, const 
   int dev = -1;
   CUDA_TRY(nullptr, cudaGetDevice(&dev));
   if (dev < 0 || dev >= TIDAR_STATIC_MAX_DEVICES) return fail(nullptr, TIDAR_EINVAL, "tidar_attention_static: device ordinal %d not supported", dev);
-  if (!g_static_ptr[dev]) {                    // first call on this device: resolve the table's device address
+  // First call on this device: resolve the table's device address.  Not synchronised between
+  // host threads: two first calls at once both look the address up and store the same value.
+  if (!g_static_ptr[dev]) {
     int32_t *p = nullptr;
     CUDA_TRY(nullptr, cudaGetSymbolAddress((void **)&p, g_static_rowmeta));
     if (!p) return fail(nullptr, TIDAR_ECUDA, "tidar_attention_static: no device address for the built-in table");
@@ -1056,8 +1260,8 @@ extern "C" int tidar_attention_static(const void *q, const void *k_pages, const 
   m.loc0 = base + 3 * TIDAR_STATIC_MAX_ROWS; m.nloc = base + 4 * TIDAR_STATIC_MAX_ROWS;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // every entry a row reads is rewritten here for rows [0, R): nothing has to start at zero
-  attn_meta_kernel<<<(R + 127) / 128, 128, 0, st>>>(m, seq_len, k, R);
-  KvGeom g{n_kv_heads, head_dim, 64, pages_per_seq, page_table};
+  attn_meta_kernel<<<(R + 127) / 128, 128, 0, st>>>(m, seq_len, k, R, pages_per_seq * 64 - k);
+  KvGeom g{n_kv_heads, head_dim, 64, pages_per_seq, page_table, n_pages};
   const float scale = 1.0f / sqrtf((float)head_dim);
   dim3 grid(R, n_q_heads);
   if (head_dim == 128)

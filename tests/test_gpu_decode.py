@@ -7,6 +7,7 @@ import torch
 
 from oracle import tidar_oracle as O
 from tests.helpers import MARGIN, TOL_LOGITS, make_model, oracle_cfg, prompt_ids, top1_margin
+from tidar_synth import CONFIGS as CONFIGS_, gen_model_weights as gen_model_weights_
 
 pytestmark = pytest.mark.gpu
 
@@ -14,9 +15,16 @@ IMPLS = [0, 1]
 
 
 def _gpu(sh, wt, impl, k_max=None, debug=1, max_batch=1, max_seq_len=512):
+    """A context whose arena is followed by 64 KiB of sentinel bytes; _close() checks them."""
     from paper_2511_08923_b200 import Tidar, pack_weights
     packed = pack_weights(wt, "cuda:0")
-    return Tidar(sh, packed, k_max=k_max or sh.k, max_batch=max_batch, max_seq_len=max_seq_len, debug=debug, impl=impl)
+    return Tidar(sh, packed, k_max=k_max or sh.k, max_batch=max_batch, max_seq_len=max_seq_len, debug=debug, impl=impl,
+                 guard_bytes=64 * 1024)
+
+
+def _close(t):
+    assert t.arena_guard_intact(), "a kernel wrote past the end of the arena"
+    t.close()
 
 
 @pytest.fixture(scope="module", params=[True, False], ids=["tied", "untied"])
@@ -88,7 +96,7 @@ def test_tiny_prefill_and_teacher_forced_steps(tiny, impl):
             assert Ls[0] == so.L and toks[0] == so.emitted
         elif Ls[0] != so.L:                   # a low-margin row flipped: the two states part ways here
             break
-    t.close()
+    _close(t)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -111,33 +119,62 @@ def test_tiny_free_running_generation_matches_ar(tiny, impl):
     assert out[:upto] == ar[:upto]
     assert all(1 <= L <= k for L in Ls)
     assert t.seq_len(0) == len(prompt) + sum(Ls)
-    t.close()
+    _close(t)
+
+
+def _drive_pattern(t, sh, prompt, k, first_block0, pattern):
+    """Builds, slot by slot, a draft block whose draft i agrees (pattern[i-1]) or disagrees with
+    the verified prediction given the slots before it, then runs the natural step on it."""
+    block = [first_block0]
+    for i in range(1, k):
+        t.prefill(0, prompt, k)
+        t.set_block(0, block + [sh.mask_token_id] * (k - len(block)))
+        toks_i, _ = t.step([0], forced=[i])
+        tgt = toks_i[0][-1]                          # verified prediction after i slots
+        block.append(tgt if pattern[i - 1] else (tgt + 1) % (sh.vocab - 1))
+    t.prefill(0, prompt, k)
+    t.set_block(0, block)
+    toks, L = t.step([0])
+    expect = next((i for i, ok in enumerate(pattern) if not ok), k - 1) + 1
+    assert L[0] == expect, (pattern, block)
+    assert toks[0][:expect - 1] == block[1:expect]
+    targets = t.argmax(0, k)                         # the step's own argmax ids of the causal slots
+    assert L[0] == O.accept_length(block, targets) and toks[0][-1] == int(targets[expect - 1])
+    return block, L[0]
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-def test_acceptance_scan_all_patterns(tiny, impl):
-    """Every agree/disagree pattern of the k-1 drafts, driven through the real step."""
+@pytest.mark.parametrize("k", [4, 8])
+def test_acceptance_scan_all_patterns(tiny, impl, k):
+    """Every agree/disagree pattern of the k-1 drafts, driven through the real step (k = 4 and 8)."""
     sh, wt, cfg, w, prompt = tiny
-    k = sh.k
-    t = _gpu(sh, wt, impl, debug=0)
-    first = t.prefill(0, prompt, k)
-    blk = t.get_block(0, k)
+    t = _gpu(sh, wt, impl, k_max=k, debug=0)
+    t.prefill(0, prompt, k)
+    b0 = t.get_block(0, k)[0]
     for pattern in itertools.product([True, False], repeat=k - 1):
-        # targets of causal slot 0 do not depend on drafts; build slot by slot
-        block = [blk[0]]
-        for i in range(1, k):
-            t.prefill(0, prompt, k)
-            t.set_block(0, block + [sh.mask_token_id] * (k - len(block)))
-            toks_i, L_i = t.step([0], forced=[i])
-            tgt = toks_i[0][-1]                          # verified prediction after i slots
-            block.append(tgt if pattern[i - 1] else (tgt + 1) % (sh.vocab - 1))
-        t.prefill(0, prompt, k)
-        t.set_block(0, block)
-        toks, L = t.step([0])
-        expect = next((i for i, ok in enumerate(pattern) if not ok), k - 1) + 1
-        assert L[0] == expect, (pattern, block)
-        assert toks[0][:expect - 1] == block[1:expect]
-    t.close()
+        _drive_pattern(t, sh, prompt, k, b0, pattern)
+    _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("k", [16, 32])
+def test_acceptance_scan_wide_blocks(tiny, impl, k):
+    """k = 16 and k = 32 (every lane of the verifying warp in use at 32): all drafts agree, the
+    first disagrees, only the last disagrees, and a seeded sample of mixed patterns."""
+    sh, wt, cfg, w, prompt = tiny
+    t = _gpu(sh, wt, impl, k_max=k, debug=0, max_seq_len=256)
+    t.prefill(0, prompt, k)
+    b0 = t.get_block(0, k)[0]
+    rng = np.random.default_rng(k)
+    patterns = [tuple([True] * (k - 1)), tuple([False] + [True] * (k - 2)), tuple([True] * (k - 2) + [False]),
+                tuple([True] * (k // 2) + [False] * (k - 1 - k // 2))]
+    patterns += [tuple(bool(x) for x in rng.random(k - 1) < 0.85) for _ in range(4 if k == 16 else 2)]
+    seen = set()
+    for pattern in patterns:
+        _, L = _drive_pattern(t, sh, prompt, k, b0, pattern)
+        seen.add(L)
+    assert k in seen and 1 in seen and (k - 1) in seen
+    _close(t)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -158,7 +195,7 @@ def test_forced_acceptance_and_poisoned_eviction(tiny, impl):
         assert n == len(prompt) + 11
         rec.append([t.kv(0, l, 0, n) for l in range(cfg.n_layers)])
         runs.append(rec)
-        t.close()
+        _close(t)
     for a, b in zip(runs[0][:-1], runs[1][:-1]):
         assert a[0] == b[0] and a[1] == b[1]
         np.testing.assert_array_equal(a[2], b[2])
@@ -196,7 +233,7 @@ def test_committed_kv_is_exact_and_never_rewritten(tiny, impl):
     t2.prefill(0, seq[:n_final], k)
     k0, v0 = t2.kv(0, 0, 0, n_final)
     np.testing.assert_array_equal(k0, final[0][0]); np.testing.assert_array_equal(v0, final[0][1])
-    t.close(); t2.close()
+    _close(t); _close(t2)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -210,7 +247,7 @@ def test_batched_step_equals_single_sequence_steps(impl):
         out = [t.prefill(0, p, k)]
         for L in (2, 1, 4):
             out.extend(t.step([0], forced=[L])[0][0])
-        single.append(out); t.close()
+        single.append(out); _close(t)
     t = _gpu(sh, wt, impl, debug=0, max_batch=3)
     outs = [[t.prefill(i, p, k)] for i, p in enumerate(prompts)]
     for L in (2, 1, 4):
@@ -218,7 +255,7 @@ def test_batched_step_equals_single_sequence_steps(impl):
         for i in range(3):
             outs[i].extend(toks[i])
     assert outs == single
-    t.close()
+    _close(t)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -241,7 +278,7 @@ def test_errors_are_reported_before_launch(impl):
         t.prefill(0, [5000], 4)
     with pytest.raises(TidarError):
         t.step([0], forced=[9])
-    t.close()
+    _close(t)
 
 
 @pytest.mark.parametrize("name,over", [
@@ -268,4 +305,79 @@ def test_other_shapes_prefill_and_steps(name, over):
         toks, Ls = t.step([0], forced=[3])
         _compare_pass(t, so.fwd, np.arange(k * (k + 1)))
         assert Ls == [3]
-    t.close()
+    _close(t)
+
+
+@pytest.mark.parametrize("name", ["tiny", "1.5b", "8b"])
+def test_graph_replay_plain_launches_and_replay_kernels_agree(name):
+    """The benchmark times the captured-graph path with programmatic dependent launches; the
+    logits / hidden-state comparisons run with plain launches.  The same teacher-forced steps
+    through (a) graph replay, (b) plain launches and (c) the fp32 CUDA-core kernels must give
+    identical acceptance lengths, tokens and next blocks, and (a) and (b) bit-identical cached
+    K/V in every layer (same kernels, same order: a kernel that read its input before the
+    previous kernel finished would show here)."""
+    from dataclasses import replace
+    if name == "tiny":
+        sh, k, n_prompt = CONFIGS_["tiny"], 4, 64
+    else:
+        sh = replace(CONFIGS_[name].reduced(2), vocab=8192)          # the benchmark's widths, two layers, small head
+        k, n_prompt = 16, 200
+    wt = gen_model_weights_(sh)
+    prompt = prompt_ids(sh, n_prompt)
+    forced = [3, k, 1, k // 2, 2]
+    runs = {}
+    for tag, impl, debug in (("graph", 0, 0), ("plain", 0, 8), ("replay", 1, 0)):
+        t = _gpu(sh, wt, impl, k_max=k, debug=debug, max_seq_len=n_prompt + 8 * k + 64)
+        rec = [t.prefill(0, prompt, k)]
+        blocks = [t.get_block(0, k)]
+        for f in forced:
+            if tag != "graph":
+                t.set_block(0, runs["graph"]["blocks"][len(rec) - 1])          # teacher-forced from run (a)
+            toks, L = t.step([0], forced=[f])
+            rec.append((toks[0], L[0]))
+            blocks.append(t.get_block(0, k))
+        n = t.seq_len(0)
+        kv = [t.kv(0, l, 0, n) for l in range(sh.n_layers)] if impl == 0 else None
+        runs[tag] = {"rec": rec, "blocks": blocks, "kv": kv, "n": n, "launches": t.launch_count()}
+        _close(t)
+    assert runs["graph"]["rec"] == runs["plain"]["rec"] and runs["graph"]["blocks"] == runs["plain"]["blocks"]
+    assert runs["graph"]["n"] == runs["plain"]["n"]
+    for (k0, v0), (k1, v1) in zip(runs["graph"]["kv"], runs["plain"]["kv"]):
+        np.testing.assert_array_equal(k0, k1); np.testing.assert_array_equal(v0, v1)
+    # the CUDA-core kernels round differently: tokens can only differ on a near-tie, which the
+    # tiny model's margins make rare; lengths are forced, so the shapes must match exactly
+    assert [r[1] for r in runs["replay"]["rec"][1:]] == [r[1] for r in runs["graph"]["rec"][1:]]
+    same = sum(a == b for a, b in zip(runs["replay"]["rec"], runs["graph"]["rec"]))
+    assert same >= len(forced), (runs["replay"]["rec"], runs["graph"]["rec"])
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_device_timeout_status_is_reported_and_sequences_released(tiny, impl):
+    """The status word a kernel sets when one of its bounded waits gives up reaches the caller as
+    TIDAR_EDEVICE_TIMEOUT, and the sequences of the failed step must be prefilled again.  The word
+    is set through a debug hook: no kernel is made to wait."""
+    from paper_2511_08923_b200 import TidarError
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    t = _gpu(sh, wt, impl, debug=0)
+    t.prefill(0, prompt, k)
+    t.step([0], forced=[2])
+    if impl != 0:                                   # the replay kernels have no bounded waits and no status word to read
+        _close(t)
+        return
+    t.force_status(2)
+    with pytest.raises(TidarError) as e:
+        t.step([0], forced=[1])
+    assert e.value.code == -5
+    with pytest.raises(TidarError) as e:            # released: not prefilled any more
+        t.step([0], forced=[1])
+    assert e.value.code == -1
+    first = t.prefill(0, prompt, k)                 # and usable again
+    toks, L = t.step([0], forced=[2])
+    assert L == [2]
+    t.force_status(1)
+    with pytest.raises(TidarError) as e:
+        t.sync()
+    assert e.value.code == -5
+    t.sync()                                        # the word was cleared by the report
+    _close(t)

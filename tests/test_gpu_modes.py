@@ -1,0 +1,163 @@
+"""Autoregressive mode, likelihood scoring, per-step block length and beta < 1 on the GPU
+(needs a B200): every entry point through the C ABI against the oracle."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch  # noqa: F401
+
+from oracle import tidar_oracle as O
+from tests.helpers import MARGIN, TOL_LOGITS, make_model, oracle_cfg, prompt_ids, top1_margin
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [0, 1]
+
+
+def _gpu(sh, wt, impl, k_max, debug=0, max_batch=1, max_seq_len=512, beta=1.0):
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    return Tidar(sh, pack_weights(wt, "cuda:0"), k_max=k_max, max_batch=max_batch, max_seq_len=max_seq_len, debug=debug, impl=impl,
+                 guard_bytes=64 * 1024, beta=beta)
+
+
+def _close(t):
+    assert t.arena_guard_intact()
+    t.close()
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    sh, wt = make_model("tiny", tied=False)
+    return sh, wt, oracle_cfg(sh), O.weights_to_f64(wt), prompt_ids(sh)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_autoregressive_steps_match_plain_greedy_decoding(tiny, impl):
+    """tidar_ar_step (one causal slot, no mask slots) against the oracle's one-token-per-pass decoder."""
+    sh, wt, cfg, w, prompt = tiny
+    n_new = 24
+    ar = O.ar_generate(cfg, w, prompt, n_new)
+    t = _gpu(sh, wt, impl, k_max=4)
+    first = t.prefill(0, prompt, 1)
+    fo = O.causal_forward(cfg, w, list(prompt) + ar)
+    m = top1_margin(fo.logits[len(prompt) - 1:len(prompt) - 1 + n_new])      # margin of the prediction of new token i
+    if m[0] > MARGIN:
+        assert first == ar[0]
+    launches0 = t.launch_count()
+    checked = 0
+    for i in range(n_new - 1):                      # teacher-forced with the oracle's tokens: the caches stay comparable
+        t.set_block(0, [ar[i]])
+        nxt = t.ar_step([0])
+        if m[i + 1] > MARGIN:
+            assert nxt == [ar[i + 1]], (i, nxt, ar[i + 1])
+            checked += 1
+    assert checked >= n_new // 2
+    per_step = (t.launch_count() - launches0) / (n_new - 1)
+    assert t.seq_len(0) == len(prompt) + n_new - 1
+    # the committed cache is the one a causal pass over the same tokens gives
+    from paper_2511_08923_b200 import bf16_bits_to_f32
+    n = t.seq_len(0)
+    for l in range(cfg.n_layers):
+        kk, vv = t.kv(0, l, 0, n)
+        assert np.abs(bf16_bits_to_f32(kk) - fo.k_new[l][:n]).max() <= TOL_LOGITS
+        assert np.abs(bf16_bits_to_f32(vv) - fo.v_new[l][:n]).max() <= TOL_LOGITS
+    # a TiDAR step after autoregressive steps finds no drafts: it accepts one token and leaves a full block
+    toks, L = t.step_k([0], 4)
+    assert L == [1] and len(t.get_block(0, 4)) == 4
+    toks2, L2 = t.step([0])
+    assert 1 <= L2[0] <= 4
+    assert per_step < 60, per_step            # one slot per sequence: no mask-slot work
+    _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_likelihood_scoring_matches_causal_log_softmax(tiny, impl):
+    """tidar_score: log p(next token) of every position from one causal pass (the model's
+    autoregressive mode), against log-softmax of the oracle's causal logits; also across chunks."""
+    sh, wt, cfg, w, prompt = tiny
+    rng = np.random.default_rng(5)
+    for n in (2, 37, 300):                          # 300 rows: more than one chunk of the row capacity
+        ids = rng.integers(0, sh.vocab - 1, n)
+        fo = O.causal_forward(cfg, w, ids)
+        lg = fo.logits[:-1]
+        lse = np.log(np.exp(lg - lg.max(-1, keepdims=True)).sum(-1)) + lg.max(-1)
+        want = lg[np.arange(n - 1), ids[1:]] - lse
+        t = _gpu(sh, wt, impl, k_max=4)
+        got = t.score(0, ids)
+        assert got.shape == (n - 1,)
+        assert np.abs(got - want).max() <= TOL_LOGITS, np.abs(got - want).max()
+        # the slot was scratch: nothing is left in it, and it can be prefilled afterwards
+        from paper_2511_08923_b200 import TidarError
+        with pytest.raises(TidarError):
+            t.step([0])
+        t.prefill(0, prompt, 4); t.step([0])
+        _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_block_length_chosen_per_step(tiny, impl):
+    """tidar_step_k: shorter and longer blocks than the previous pass left.  Greedy TiDAR with beta = 1
+    emits the autoregressive continuation whatever the block lengths are; a step that asks for more
+    drafts than the sequence holds feeds mask tokens for the missing ones and never accepts them."""
+    sh, wt, cfg, w, prompt = tiny
+    n_new = 40
+    ar = O.ar_generate(cfg, w, prompt, n_new + 8)
+    fo = O.causal_forward(cfg, w, list(prompt) + ar)
+    m = top1_margin(fo.logits[len(prompt) - 1:len(prompt) - 1 + n_new])
+    unsure = np.nonzero(m <= MARGIN)[0]
+    upto = int(unsure[0]) if len(unsure) else n_new
+    t = _gpu(sh, wt, impl, k_max=8, max_seq_len=256)
+    out = [t.prefill(0, prompt, 4)]
+    held = 4
+    for k in (2, 8, 8, 3, 1, 5, 8, 4, 4, 8, 8, 8):
+        toks, L = t.step_k([0], k)
+        assert 1 <= L[0] <= min(k, held), (k, held, L)         # only drafts the sequence holds can be accepted
+        out.extend(toks[0]); held = k
+        assert t.seq_len(0) == len(prompt) + len(out) - 1
+        if len(out) >= n_new:
+            break
+    assert out[:upto] == ar[:upto]
+    assert t.ridge_k(1) == 8 and t.ridge_k(4) == 8 and t.ridge_k(8, 288) == 5 and t.ridge_k(32, 288) == 2 and t.ridge_k(1000) == 1
+    _close(t)
+
+
+# ---- beta < 1 ------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("beta", [0.0, 0.5])
+def test_beta_mixed_verification(tiny, impl, beta):
+    """beta < 1 (paper Section 4.4.3): drafts are verified against argmax(beta * logits_ar + (1 - beta) *
+    logits_diff).  beta = 0 trusts the diffusion prediction alone: the verified targets must equal the
+    argmax of the first slot of each block, which the GPU also reports on its own rows."""
+    sh, wt, cfg, w, prompt = tiny
+    k = sh.k
+    cfg_b = replace(cfg, beta=beta)
+    t = _gpu(sh, wt, impl, k_max=k, debug=1, beta=beta)
+    first = t.prefill(0, prompt, k)
+    st, c, fo = O.prefill(cfg_b, w, prompt, k, return_forward=True)
+    n = len(prompt)
+    mixed = beta * fo.logits[n - 1] + (1 - beta) * fo.logits[n]
+    if top1_margin(mixed) > MARGIN:
+        assert first == c
+    T = k * (k + 1)
+    for s in range(4):
+        t.set_block(0, st.block)
+        block = st.block.copy()
+        so = O.step(cfg_b, w, st)
+        toks, L = t.step([0])
+        n_rows, _ = t.last_rows()
+        assert n_rows == T + k                      # the k mixed rows follow the slots
+        lg = t.logits(0, n_rows)
+        ids = t.argmax(0, n_rows)
+        ref_mixed = beta * so.fwd.logits[:k] + (1 - beta) * so.fwd.logits[k:].reshape(k, k, -1)[:, 0, :]
+        assert np.abs(lg[:T] - so.fwd.logits).max() <= TOL_LOGITS
+        assert np.abs(lg[T:] - ref_mixed).max() <= TOL_LOGITS          # mixing the LM head's input rows = mixing the logits
+        tg = ids[T:]
+        if beta == 0.0:                             # the diffusion prediction alone
+            np.testing.assert_array_equal(lg[T:].argmax(-1), lg[k:T:k].argmax(-1))
+        L_ref = O.accept_length(block, tg)
+        assert L[0] == L_ref and toks[0] == [int(x) for x in block[1:L_ref]] + [int(tg[L_ref - 1])]
+        if (top1_margin(ref_mixed) > MARGIN).all():
+            assert L[0] == so.L and toks[0] == so.emitted
+        elif L[0] != so.L:
+            break
+    _close(t)

@@ -18,3 +18,4 @@ from .generators import (  # noqa: F401
     tensor_id,
     uniform01,
 )
+from .lazy import LazyLayers, LazyRows, lazy_model_weights, production_seconds  # noqa: F401

@@ -167,13 +167,15 @@ CONFIGS: Dict[str, ModelShape] = {
 }
 
 
-def gen_model_weights(shape: ModelShape, device="cpu", layers=None) -> dict:
+def gen_model_weights(shape: ModelShape, device="cpu", layers=None, with_head: bool = True) -> dict:
     """bf16 weights for ``shape``; matrices are [out_features, in_features].
 
     Norm gains are 1 + N(0, 0.1^2), rounded to bf16, so that a kernel that
     drops or misplaces a gain cannot pass.
     ``layers`` restricts generation to a subset of layer indices (the rest are
-    left out of the returned list), for bounded CPU samples of a big model.
+    left out of the returned list), for bounded CPU samples of a big model;
+    ``with_head=False`` leaves out the embedding, the LM head and the final norm
+    (for callers that fetch a big model one layer at a time).
     """
     s, d, hd = shape.seed, shape.d_model, shape.head_dim
     std = shape.init_std
@@ -185,9 +187,11 @@ def gen_model_weights(shape: ModelShape, device="cpu", layers=None) -> dict:
         g = gen_normal_bf16(s, tensor_id(kind, layer), d, 0.1, device).to(torch.float32)
         return (1.0 + g).to(torch.bfloat16)
 
-    w = {"embed": mat("embed", 0, shape.vocab, d),
-         "final_norm": gain("final_norm", 0)}
-    w["lm_head"] = w["embed"] if shape.tie_lm_head else mat("lm_head", 0, shape.vocab, d)
+    w = {}
+    if with_head:
+        w = {"embed": mat("embed", 0, shape.vocab, d),
+             "final_norm": gain("final_norm", 0)}
+        w["lm_head"] = w["embed"] if shape.tie_lm_head else mat("lm_head", 0, shape.vocab, d)
     w["layers"] = []
     for l in (range(shape.n_layers) if layers is None else layers):
         w["layers"].append({
