@@ -114,47 +114,37 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------
-# CPU oracle on a bounded sample
+# CPU oracle: one whole decode step, timed
 # ----------------------------------------------------------------------------
-def oracle_sample(sh, k, n, with_head=True, rows=None):
-    """Time the oracle on ONE layer (+ the LM head) of one decode step; extrapolate a step.
+def oracle_step_timed(sh, k, n, n_steps=1):
+    """Times `n_steps` full decode steps of the CPU oracle (every layer, the whole LM head, acceptance,
+    selection, commit) for one sequence with n cached positions.
 
-    The weights are the generator's (layer 0 and the LM head); the embedding table is
-    restricted to the ids in use (ids remapped), the cache holds seeded random K/V.
+    The oracle runs as it stands (float64 NumPy on the host cores).  Its weights are the generator's,
+    handed over one layer at a time (produced on the GPU when there is one, else on the host) so that
+    the host never holds more than one layer in float64; the time spent producing them is measured
+    and NOT counted.  The cache holds seeded random K/V (timing does not depend on the values).
+    Returns (seconds per step, seconds spent producing weights per step).
     """
     from oracle import tidar_oracle as O
+    from tidar_synth import lazy_model_weights, production_seconds
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    w = gen_model_weights(sh.reduced(1), device=dev)
-    lay = {kk: (vv if kk == "index" else vv.cpu()) for kk, vv in w["layers"][0].items()}
-    block = gen_token_ids(sh.seed, tensor_id("drafts"), k, sh.vocab - 1).numpy().astype(np.int64)
-    used = np.unique(np.concatenate([block, [sh.mask_token_id]]))
-    remap = {int(u): i for i, u in enumerate(used)}
-    small_embed = w["embed"][torch.as_tensor(used, device=w["embed"].device)].cpu()
-    wd = {"embed": small_embed, "final_norm": w["final_norm"].cpu(), "lm_head": w["lm_head"].cpu(), "layers": [lay]}
-    t0 = time.perf_counter()
-    w64 = O.weights_to_f64(wd)
-    t_upcast = time.perf_counter() - t0
-    cfg = O.OracleConfig(1, sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.d_ffn, sh.vocab, sh.rope_theta,
-                         sh.rms_eps, remap[sh.mask_token_id], 1.0)
+    w = lazy_model_weights(sh, dev)
+    cfg = O.OracleConfig(sh.n_layers, sh.d_model, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.d_ffn, sh.vocab, sh.rope_theta,
+                         sh.rms_eps, sh.mask_token_id, 1.0)
     rng = np.random.default_rng(sh.seed)
-    st = O.OracleState(n=n, k_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim))],
-                       v_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim))],
-                       block=np.array([remap[int(b)] for b in block]))
-    # layer part: a pass without the head (logit_rows empty), head part: the difference
-    T = k * (k + 1)
-    _, _, _, pos = O.slot_layout(n, k)
-    ids = np.concatenate([st.block, np.full(k * k, cfg.mask_token_id, dtype=np.int64)])
-    mask = O.build_decode_mask(n, k)
-
-    def run(head):
+    block = gen_token_ids(sh.seed, tensor_id("drafts"), k, sh.vocab - 1).numpy().astype(np.int64)
+    st = O.OracleState(n=n, k_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim)) for _ in range(sh.n_layers)],
+                       v_cache=[rng.standard_normal((n, sh.n_kv_heads, sh.head_dim)) for _ in range(sh.n_layers)], block=block)
+    total, gen = 0.0, 0.0
+    for _ in range(n_steps):
+        g0 = production_seconds()
         t0 = time.perf_counter()
-        O.forward(cfg, w64, ids, pos, mask, st.k_cache, st.v_cache, logit_rows=None if head else np.array([], dtype=np.int64))
-        return time.perf_counter() - t0
-    return run, t_upcast
-
-
-def oracle_step_seconds(sh, t_layer, t_head):
-    return sh.n_layers * t_layer + t_head
+        O.step(cfg, w, st)
+        dt = time.perf_counter() - t0
+        dg = production_seconds() - g0
+        total += dt - dg; gen += dg
+    return total / n_steps, gen / n_steps
 
 
 def blas_threads():
@@ -168,43 +158,28 @@ def blas_threads():
 
 # ----------------------------------------------------------------------------
 def run_reference(args, sh, k, n0):
+    """The reference arm: the CPU oracle on this workload.  A full 8B-class oracle step takes ~10 s of
+    float64 arithmetic, so the arm times a bounded number of whole steps (one by default) whatever
+    --steps says, and reports that number as `steps`."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sched = acceptance_schedule(SCHEDULE_SEED, args.steps + args.warmup, k).numpy()
-    run, _ = oracle_sample(sh, k, n0)
-    t_l = run(False)
-    t_full = run(True)
-    t_h = max(t_full - t_l, 0.0)
-    budget = 150.0
-    total_steps = args.steps + args.warmup
-    do_head = total_steps * (t_l + t_h) <= budget
-    layer_s, head_s = [], []
-    for s in range(total_steps):
-        if do_head:
-            a = run(False); b = run(True)
-            if s >= args.warmup:
-                layer_s.append(a); head_s.append(max(b - a, 0.0))
-        elif total_steps * t_l <= budget:
-            a = run(False)
-            if s >= args.warmup:
-                layer_s.append(a); head_s.append(t_h)
-        else:
-            if s >= args.warmup:
-                layer_s.append(t_l); head_s.append(t_h)
-    step_s = [oracle_step_seconds(sh, a, b) for a, b in zip(layer_s, head_s)]
-    L = sched[args.warmup:]
-    value = float(L.sum() / sum(step_s))
-    sample = (f"per step: one of {sh.n_layers} layers" + (" + the full LM head" if do_head else " (LM head timed once)") +
-              f" of one decode step (k={k}, {k*(k+1)} slots, n={n0}); step time = n_layers*layer + head")
-    if not do_head and total_steps * t_l > budget:
-        sample = "calibration pass only (one layer + LM head timed once; requested steps exceed the time bound); " + sample
+    n_timed = max(1, min(args.steps, args.ref_steps))
+    step_s, gen_s = oracle_step_timed(sh, k, n0, n_timed)
+    mean_L = float(acceptance_schedule(SCHEDULE_SEED, 4096, k).numpy().mean())
+    value = mean_L / step_s
     cores = blas_threads()
+    sample = (f"{n_timed} whole decode step(s) of the unmodified oracle (all {sh.n_layers} layers, full LM head, k={k}, {k*(k+1)} slots, "
+              f"n={n0} cached positions, float64 NumPy); weights handed over layer by layer, their production "
+              f"({gen_s:.1f} s per step) not counted; tokens/s = mean schedule acceptance {mean_L:.2f} / step time")
+    cfgd = workload_config(sh, k, n0, 1)
+    cfgd["reference_steps_timed"] = n_timed
+    cfgd["reference_steps_requested"] = args.steps
     line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(step_s) / len(step_s),
+            "steps": n_timed, "warmup": 0, "ms_per_step": 1e3 * step_s,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(sh, k, n0, 1),
-            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "config": cfgd, "extrapolated": False,
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample, "extrapolated": False},
             "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -237,12 +212,99 @@ def attention_microbench(reps=50):
             t.attention(q, kp, vp, pt, sl, kl, vl, out, 1, k)
         e1.record(); torch.cuda.synchronize()
         us = e0.elapsed_time(e1) / reps * 1e3
+        # skipped-tile evidence: key tiles the kernel's CTAs visit in one call, against a dense mask
+        # (every 128-row query tile of every KV head against every 64-key tile of [cache | step slots])
+        t.count_attention_tiles(True)
+        t.attention(q, kp, vp, pt, sl, kl, vl, out, 1, k)
+        visited = t.count_attention_tiles(False)
+        spt = 128 // (Hq // Hkv)
+        q_tiles = (T + spt - 1) // spt
+        dense = Hkv * q_tiles * ((n + k + 63) // 64 + (k * k + 63) // 64)
+        local_blocks = (2 * k + 1) / float((k + 1) ** 2)
+        # the cached part is dense for every row; what the mask's block structure saves is in the step-local part
+        cache_tiles = 0
+        for qt in range(q_tiles):
+            slots = range(qt * spt, min((qt + 1) * spt, T))
+            nvis = max(n + s_ + 1 if s_ < k else n + (s_ - k) // k + 1 for s_ in slots)
+            cache_tiles += (nvis + 63) // 64
+        local_visited = visited - Hkv * cache_tiles
+        local_dense = Hkv * q_tiles * ((k * k + 63) // 64)
         keys = sum(n + j + 1 for j in range(k)) + sum(k * (n + b + 1 + k) for b in range(k))
         flops, nbytes = 4 * Hq * hd * keys, n * Hkv * hd * 2 * 2
         print(json.dumps({"attention_microbench": {"cached_positions": n, "k": k, "heads": f"{Hq}/{Hkv}", "head_dim": hd},
                           "us_per_call": round(us, 1), "tflops": round(flops / us / 1e6, 1), "kv_gbs": round(nbytes / us / 1e3, 1),
-                          "frac_of_measured_bf16_peak": round(flops / us / 1e6 / pk["bf16_tflops_sustained"], 3)}))
+                          "frac_of_measured_bf16_peak": round(flops / us / 1e6 / pk["bf16_tflops_sustained"], 3),
+                          "key_tiles_visited": visited, "key_tiles_dense_mask": dense, "skipped_tile_frac": round(1.0 - visited / dense, 4),
+                          "local_tiles_visited": local_visited, "local_tiles_dense_mask": local_dense,
+                          "local_skipped_tile_frac": round(1.0 - local_visited / local_dense, 4),
+                          "local_kxk_subblocks_nonempty_frac": round(local_blocks, 4)}))
     t.close()
+
+
+def measure_classes(t, seqs, forced_L, impl, n_t=4):
+    """Per-class kernel time of a step (ms): (timeline in graph mode, CUDA events around plain launches)."""
+    cls, cls_plain = {}, {}
+    if impl == 0:
+        t.set_timeline(True)
+        t.step(seqs, forced_L)                        # re-captures the graph with the stamps in
+        for _ in range(n_t):
+            t.step(seqs, forced_L)
+            for kk, v in t.timeline().items():
+                cls[kk] = cls.get(kk, 0.0) + v / n_t
+        t.set_timeline(False)
+    t.set_timing(True)
+    for _ in range(n_t):
+        t.step(seqs, forced_L)
+        for kk, v in t.timing().items():
+            cls_plain[kk] = cls_plain.get(kk, 0.0) + v / n_t
+    t.set_timing(False)
+    if not cls:
+        cls = dict(cls_plain)
+    return cls, cls_plain
+
+
+def measure_other_workload(sh, impl, dev, stream, steps=64, warmup=5):
+    """One more model class in the same run: build it, prefill, time `steps` decode steps under the
+    schedule (CUDA events on the library's stream), per-class kernel time, roofline fractions."""
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    k, n0 = sh.k, sh.prompt_len
+    packed = pack_weights(gen_model_weights(sh, device=dev), dev)
+    t = Tidar(sh, packed, k_max=k, max_batch=1, max_seq_len=n0 + (steps + warmup + 16) * k + 64, impl=impl, device=dev, stream=stream)
+    prompt = gen_token_ids(sh.seed, tensor_id("prompt"), n0, sh.vocab - 1).numpy()
+    t.prefill(0, prompt, k)
+    sched = acceptance_schedule(SCHEDULE_SEED, steps + warmup, k).numpy()
+    for i in range(warmup):
+        t.step_async([0], [int(sched[i])]); t.step_wait()
+    n_start = t.seq_len(0)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    tokens = 0
+    for i in range(steps):
+        t.step_async([0], [int(sched[warmup + i])]); _, L = t.step_wait(); tokens += sum(L)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    n_mid = (n_start + t.seq_len(0)) // 2
+    cls, _ = measure_classes(t, [0], [8], impl)
+    t.close()
+    pk, pk_src = peaks()
+    cost = step_cost(sh, k, n_mid)
+    t_hbm = cost["bytes"] / (pk["hbm_gbs"] * 1e9) * 1e3
+    t_tensor = cost["flops"] / (pk["bf16_tflops_sustained"] * 1e12) * 1e3
+    gemm_ms = cls.get("gemm", 0.0) + cls.get("lmhead", 0.0)
+    return {"config": workload_config(sh, k, n0, 1), "steps": steps, "warmup": warmup, "ms_per_step": ms, "tokens_per_s": tokens / (ms * steps) * 1e3,
+            "mean_accept_len": tokens / steps,
+            "step_roofline": {"bytes": cost["bytes"], "flops": cost["flops"], "n_cached": n_mid, "t_hbm_ms": t_hbm, "t_tensor_ms": t_tensor,
+                              "frac_measured_peaks": max(t_hbm, t_tensor) / ms,
+                              "frac_nominal_peaks": max(cost["bytes"] / (NOMINAL["hbm_gbs"] * 1e9), cost["flops"] / (NOMINAL["bf16_tflops"] * 1e12)) * 1e3 / ms,
+                              "peak_source": pk_src},
+            "roofline": {"bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                         "achieved": (cost["gemm_flops"] / (gemm_ms * 1e-3) / 1e12) if t_tensor >= t_hbm else (cost["weight_bytes"] / (gemm_ms * 1e-3) / 1e9),
+                         "peak": pk["bf16_tflops_sustained"] if t_tensor >= t_hbm else pk["hbm_gbs"], "unit": "TFLOP/s" if t_tensor >= t_hbm else "GB/s",
+                         "frac": ((cost["gemm_flops"] / (gemm_ms * 1e-3) / 1e12) / pk["bf16_tflops_sustained"]) if t_tensor >= t_hbm
+                                 else ((cost["weight_bytes"] / (gemm_ms * 1e-3) / 1e9) / pk["hbm_gbs"]),
+                         "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {x: round(y, 4) for x, y in cls.items()}}}
 
 
 def workload_config(sh, k, n0, batch):
@@ -269,8 +331,10 @@ def main():
     ap.add_argument("--per-l-steps", type=int, default=2)
     ap.add_argument("--ar-steps", type=int, default=32, help="steps of the k = 1 autoregressive reference (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-steps", type=int, default=1, help="whole oracle steps the reference arm / CPU baseline times (one 8B-class step is ~10 s of float64 work)")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the 1.5B-class step that the default run reports beside the 8B-class one")
     ap.add_argument("--attn-microbench", action="store_true", help="time the attention entry point alone at 1 k .. 32 k cached positions and exit")
-    ap.add_argument("--lib-debug", type=int, default=0, help="library debug bits (4: bf16 split-K partial sums; diagnostics, not the bench configuration)")
+    ap.add_argument("--lib-debug", type=int, default=0, help="library debug bits (4: bf16 split-K partial sums, 8: plain launches instead of the graph; diagnostics, not the bench configuration)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -356,15 +420,12 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
 
-    # ---- per-class kernel time (CUDA events around every launch) ---------------------
-    t.set_timing(True)
-    cls = {}
-    n_t = 4
-    for _ in range(n_t):
-        t.step(seqs, forced(0, 8 if k >= 8 else k))
-        for kk, v in t.timing().items():
-            cls[kk] = cls.get(kk, 0.0) + v / n_t
-    t.set_timing(False)
+    # ---- per-class kernel time ----------------------------------------------------------
+    # (a) in the launch mode that was just timed (replayed graph, programmatic launches): every kernel
+    #     stamps the moment its first CTA got past the previous kernel and the moment its last CTA
+    #     finished (tidar_debug_set_timeline); a class's time is the sum of those intervals;
+    # (b) plain launches, each bracketed by CUDA events (no overlap between kernels): for comparison.
+    cls, cls_plain = measure_classes(t, seqs, forced(0, 8 if k >= 8 else k), impl)
 
     # ---- per acceptance length -----------------------------------------------------------
     per_L = {}
@@ -384,10 +445,10 @@ def main():
         ms = a.elapsed_time(b) / args.per_l_steps
         per_L[str(L)] = {"ms_per_step": round(ms, 4), "tokens_per_s": round(B * L / ms * 1e3, 1)}
 
-    # ---- autoregressive reference on the same kernels: k = 1 (one settled token per pass) ----
+    # ---- autoregressive reference on the same kernels: one causal slot per pass (tidar_ar_step) ----
     # The paper's headline is decode tokens/s relative to plain AR decoding of the same model
-    # (Section 4.3); this gives the same ratio on this GPU.  A k = 1 step carries one causal slot
-    # and one mask slot and always emits exactly one token.
+    # (Section 4.3); this gives the same ratio on this GPU.  An AR step carries the settled token
+    # alone (T = 1, no mask slots) and always emits exactly one token.
     ar = None
     if args.ar_steps > 0 and B == 1:
         t.close()
@@ -395,20 +456,28 @@ def main():
                   debug=args.lib_debug)
         t.prefill(0, prompt, 1)
         for _ in range(3):
-            t.step_async([0], [1]); t.step_wait()
+            t.ar_step([0])
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record(stream)
         for _ in range(args.ar_steps):
-            t.step_async([0], [1]); t.step_wait()
+            t.ar_step([0])
         b.record(stream)
         torch.cuda.synchronize()
         ar_ms = a.elapsed_time(b) / args.ar_steps
-        ar = {"ms_per_step": round(ar_ms, 4), "tokens_per_s": round(1e3 / ar_ms, 1), "steps": args.ar_steps,
+        ar = {"ms_per_step": round(ar_ms, 4), "tokens_per_s": round(1e3 / ar_ms, 1), "steps": args.ar_steps, "slots_per_step": 1,
               "hbm_frac_of_measured_peak": None}
 
     if world > 1:
         ms_total, e2e_s, tokens, tokens_e2e = aggregate_over_ranks(ms_total, e2e_s, tokens, tokens_e2e, dev)
+    t.close()
+    t, packed = None, None
+    torch.cuda.empty_cache()
+
+    # ---- the other model class the target names (1.5B-class, k = 16): same kernels, a short run (N = 1 only) ----
+    other = None
+    if world == 1 and args.workload == "8b" and not args.layers and B == 1 and args.k is None and not args.no_other_workloads:
+        other = {"1.5b": measure_other_workload(CONFIGS["1.5b"], impl, dev, stream, steps=64)}
 
     if rank == 0:
         pk, pk_src = peaks()
@@ -435,10 +504,14 @@ def main():
         roof.update({"frac": roof["achieved"] / roof["peak"],
                      "traffic": tr["bytes_per_step"] if tr else None,
                      "traffic_note": tr["note"] if tr else "no ncu capture of this workload since the kernel last changed",
-                     "kernel": f"gemm_tc_kernel, all {n_gemm_launches} launches of one step (QKV, O, gate/up, down per layer + LM head)",
+                     "kernel": f"gemm_tc_kernel, all {n_gemm_launches} launches of one step (QKV, O, gate/up, down per layer + LM head; the class also "
+                               "holds the two small kernels that finish them: the SwiGLU fix-up of K-split tiles and the argmax merge)",
                      "algorithmic": {"flops_per_step": cost["gemm_flops"], "weight_bytes_per_step": cost["weight_bytes"]},
                      "peak_source": pk_src + (" (bf16 matmul, sustained: the kernel runs inside a long step)" if tensor_bound else " (copy bandwidth)"),
-                     "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {a: round(b, 4) for a, b in cls.items()}})
+                     "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {a: round(b, 4) for a, b in cls.items()},
+                     "timing_mode": "in-kernel %globaltimer stamps inside the replayed graph (the mode `value` is timed in): per launch, latest CTA end "
+                                    "minus earliest CTA start after its dependency; 'busy' = sum over all launches, 'span' = first start to last end",
+                     "class_ms_plain_launches": {a: round(b, 4) for a, b in cls_plain.items()}})
         line = {"metric": "decode_tokens_per_s", "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -458,16 +531,16 @@ def main():
             ar["hbm_frac_of_measured_peak"] = round(step_cost(sh, 1, n0)["bytes"] / (pk["hbm_gbs"] * 1e9) / (ar["ms_per_step"] * 1e-3), 4)
             ar["tidar_over_ar"] = round(line["value"] / ar["tokens_per_s"], 3)
             ar["paper"] = "4.71x (1.5B) / 5.91x (8B) on one H100 with trained drafts (mean acceptance 7.45 / 8.25 tokens per pass)"
-        if not args.no_cpu_baseline:
-            run, _ = oracle_sample(sh, k, n0)
-            t_l = run(False); t_f = run(True)
-            step_s = oracle_step_seconds(sh, t_l, max(t_f - t_l, 0.0))
+        if other is not None:
+            line["other_workloads"] = other
+        if not args.no_cpu_baseline and world == 1:
+            step_s, gen_s = oracle_step_timed(sh, k, n0, args.ref_steps)
             mean_L = float(sched.mean())
-            line["cpu_baseline"] = {"value": mean_L / step_s, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
-                                    "sample": f"one of {sh.n_layers} layers + the full LM head of one decode step (k={k}, n={n0}), "
-                                              f"float64 NumPy; step = n_layers*layer + head = {step_s:.1f} s"}
+            line["cpu_baseline"] = {"value": mean_L / step_s, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "extrapolated": False,
+                                    "sample": f"{args.ref_steps} whole decode step(s) of the unmodified oracle (all {sh.n_layers} layers, full LM head, "
+                                              f"k={k}, n={n0} cached positions), float64 NumPy, {step_s:.1f} s per step; weights handed over layer "
+                                              f"by layer, their production ({gen_s:.1f} s) not counted"}
         print(json.dumps(line))
-    t.close()
     if world > 1:
         dist.destroy_process_group()
 
