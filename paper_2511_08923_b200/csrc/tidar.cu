@@ -408,15 +408,16 @@ bool encode_local_map(tidar_ctx *c, CUtensorMap *tm, const void *loc, long long 
 }
 
 // Key-range split of the attention kernel: fill the SMs (two CTAs fit on one) without giving a
-// CTA fewer than two key tiles; and once half the SMs have a CTA, not fewer than five: a CTA pays
-// ~7 us of set-up, partial-result store and merge traffic whatever its key range (1.5B-class
-// step at n = 1 k: 8 splits 585 us per 4 layers, 4 splits 571), while a nearly empty machine
-// (the k = 1 step) is served best by as many CTAs as there are key tiles to hand out.
+// CTA fewer than two key tiles; and once half the SMs have a CTA, not fewer than four: a CTA pays
+// ~7 us of set-up, partial-result store and merge traffic whatever its key range, while a nearly
+// empty machine (a one-slot step) is served best by as many CTAs as there are key tiles to hand
+// out.  (8B-class heads, 1 k cached positions, 72 query-tile units: 4 splits of 4-5 tiles each
+// 26.9 us per call against 29.4 with 3 splits of 6; from 4 k positions on the limit is moot.)
 int attn_key_splits(const tidar_ctx *c, int units, int key_tiles_hint) {
   int splits = 2 * c->n_sms / std::max(units, 1);
   splits = std::min(splits, std::max(1, key_tiles_hint / 2));
   splits = std::max(1, std::min(splits, attn_tc::MAX_SPLITS));
-  while (splits > 1 && units * splits > c->n_sms / 2 && key_tiles_hint / splits < 5) --splits;
+  while (splits > 1 && units * splits > c->n_sms / 2 && key_tiles_hint / splits < 4) --splits;
   return splits;
 }
 
