@@ -307,6 +307,32 @@ def measure_other_workload(sh, impl, dev, stream, steps=64, warmup=5):
                          "launch_ms_per_step": round(gemm_ms, 4), "class_ms_per_step": {x: round(y, 4) for x, y in cls.items()}}}
 
 
+def prefill_bench(sh, impl, dev, n_prompts=(1024, 4096), reps=3):
+    """First-pass (prompt encoding) time: the default chunks of one decode step's rows against one
+    pass per prompt (`prefill_rows`), one JSON line per case.  A diagnostic beside the step benchmark."""
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    pk, _ = peaks()
+    packed = pack_weights(gen_model_weights(sh, device=dev), dev)
+    k = sh.k
+    per_layer = (sh.d_model * (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim + sh.n_q_heads * sh.head_dim * sh.d_model + 3 * sh.d_model * sh.d_ffn)
+    for n in n_prompts:
+        prompt = gen_token_ids(sh.seed, tensor_id("prompt"), n, sh.vocab - 1).numpy()
+        for rows in (0, n + k):
+            t = Tidar(sh, packed, k_max=k, max_batch=1, max_seq_len=n + 4 * k + 64, impl=impl, device=dev, prefill_rows=rows)
+            t.prefill(0, prompt, k)
+            torch.cuda.synchronize()
+            w0 = time.perf_counter()
+            for _ in range(reps):
+                t.prefill(0, prompt, k)
+            torch.cuda.synchronize()
+            ms = (time.perf_counter() - w0) / reps * 1e3
+            flops = 2.0 * (n + k) * sh.n_layers * per_layer + sum(4.0 * sh.n_q_heads * sh.head_dim * (g + 1) for g in range(n)) * sh.n_layers
+            print(json.dumps({"prefill_bench": {"workload": sh.name, "prompt_len": n, "k": k, "prefill_rows": rows or "default (rows of a decode step)"},
+                              "ms": round(ms, 2), "prompt_tokens_per_s": round(n / ms * 1e3, 1), "tflops": round(flops / ms / 1e9, 1),
+                              "frac_of_measured_bf16_peak": round(flops / ms / 1e9 / pk["bf16_tflops_sustained"], 3)}))
+            t.close()
+
+
 def workload_config(sh, k, n0, batch):
     return {"workload": f"TiDAR decode step, {sh.name}-class decoder ({sh.n_layers} layers, d_model {sh.d_model}, "
                         f"{sh.n_q_heads}/{sh.n_kv_heads} heads, head_dim {sh.head_dim}, ffn {sh.d_ffn}, vocab {sh.vocab}), "
@@ -333,6 +359,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-steps", type=int, default=1, help="whole oracle steps the reference arm / CPU baseline times (one 8B-class step is ~10 s of float64 work)")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the 1.5B-class step that the default run reports beside the 8B-class one")
+    ap.add_argument("--prefill-bench", action="store_true", help="time the first pass over 1 k and 4 k prompts, default chunks against one pass, and exit")
     ap.add_argument("--attn-microbench", action="store_true", help="time the attention entry point alone at 1 k .. 32 k cached positions and exit")
     ap.add_argument("--lib-debug", type=int, default=0, help="library debug bits (4: bf16 split-K partial sums, 8: plain launches instead of the graph; diagnostics, not the bench configuration)")
     args = ap.parse_args()
@@ -356,6 +383,9 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    if args.prefill_bench:
+        prefill_bench(sh, args.kernels if args.kernels is not None else DEFAULT_IMPL, "cuda:0")
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -80,6 +80,13 @@ typedef struct {
   int32_t impl;             /* 0: tensor-core kernels (tcgen05/TMEM/TMA);
                                1: plain fp32-accumulate CUDA-core kernels ("replay"), a
                                slow diagnostic path with the same data flow               */
+  int32_t prefill_rows;     /* rows one pass of the first pass (and of tidar_score) may carry;
+                               0 = as many as a decode step (max_batch*k_max*(k_max+1), at
+                               least 256).  With a larger value a long prompt is encoded in
+                               few passes and every weight tile, once fetched, serves all row
+                               blocks of the pass, so the first pass is bound by the tensor
+                               cores instead of re-streaming the weights per 272 rows; costs
+                               activation memory in proportion                             */
 } tidar_config;
 
 /* BORROWED device pointers.  Matrices are bf16, row-major [out_features][in_features].

@@ -35,7 +35,7 @@ class tidar_config(C.Structure):
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
                [(n, C.c_int32) for n in ("mask_token_id", "k_max", "max_batch", "max_seq_len", "page_size")] + \
                [("beta", C.c_float), ("temperature", C.c_float), ("sample_seed", C.c_uint64),
-                ("debug", C.c_int32), ("impl", C.c_int32)]
+                ("debug", C.c_int32), ("impl", C.c_int32), ("prefill_rows", C.c_int32)]
 
 
 class tidar_weights(C.Structure):
@@ -131,7 +131,7 @@ class Tidar:
 
     def __init__(self, shape, packed: dict, k_max: int, max_batch: int = 1, max_seq_len: int = 4096,
                  debug: int = 0, impl: int = 0, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
-                 guard_bytes: int = 0, beta: float = 1.0):
+                 guard_bytes: int = 0, beta: float = 1.0, prefill_rows: int = 0):
         self.lib = load()
         self.shape, self.k_max, self.max_batch = shape, k_max, max_batch
         self.device = torch.device(device)
@@ -140,7 +140,7 @@ class Tidar:
             head_dim=shape.head_dim, d_ffn=shape.d_ffn, vocab=shape.vocab, tie_lm_head=int(shape.tie_lm_head),
             rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, mask_token_id=shape.mask_token_id, k_max=k_max,
             max_batch=max_batch, max_seq_len=max_seq_len, page_size=64, beta=beta, temperature=0.0, sample_seed=0,
-            debug=debug, impl=impl)
+            debug=debug, impl=impl, prefill_rows=prefill_rows)
         self.cfg = cfg
         nbytes = C.c_size_t(0)
         rc = self.lib.tidar_arena_bytes(C.byref(cfg), C.byref(nbytes))

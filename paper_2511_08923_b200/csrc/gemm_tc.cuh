@@ -65,14 +65,22 @@ struct Args {
 };
 
 struct Item { int rb, tile, split, kb0, kb1; bool fused; };
+// Item order.  With several row blocks (a long first pass) the row block varies fastest: the CTAs
+// that run side by side then work on the SAME weight tile for different rows, so the tile comes
+// from HBM once and from L2 for the others, and the pass is bound by the tensor cores instead of
+// streaming every weight matrix once per row block.  The LM-head mode keeps a row block's tiles
+// together instead (tile fastest): its epilogue carries a running argmax per row block.
+template <int MODE>
 __device__ __forceinline__ Item decode_item(const Args &g, int item) {
   Item w;
   if (item < g.fused_items) {
-    w.fused = true; w.split = 0; w.tile = item % g.tile_b0_or_all(); w.rb = item / g.tile_b0_or_all();
+    w.fused = true; w.split = 0;
+    if (MODE == MODE_ARGMAX) { w.tile = item % g.tile_b0_or_all(); w.rb = item / g.tile_b0_or_all(); }
+    else { w.rb = item % g.n_rb; w.tile = item / g.n_rb; }
     w.kb0 = 0; w.kb1 = g.kb_total;
   } else {
     const int j = item - g.fused_items;
-    w.fused = false; w.split = j % g.S; w.tile = g.tile_b0 + (j / g.S) % g.n_tiles_b; w.rb = j / (g.S * g.n_tiles_b);
+    w.fused = false; w.rb = j % g.n_rb; w.split = (j / g.n_rb) % g.S; w.tile = g.tile_b0 + j / (g.n_rb * g.S);
     w.kb0 = (int)((long long)g.kb_total * w.split / g.S); w.kb1 = (int)((long long)g.kb_total * (w.split + 1) / g.S);
   }
   return w;
@@ -137,7 +145,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       // Weights are never written by a kernel, so nothing here waits for the previous kernel:
       // the ring fills while that kernel is still finishing.
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item w = decode_item(g, item);
+        const Item w = decode_item<MODE>(g, item);
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!sm100::mbar_wait(sm100::smem_u32(&w_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
           const uint32_t fb = sm100::smem_u32(&w_full[s]);
@@ -156,7 +164,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       pdl_wait();                      // the activations are the previous kernel's output
       tl_go(tl);
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item w = decode_item(g, item);
+        const Item w = decode_item<MODE>(g, item);
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!sm100::mbar_wait(sm100::smem_u32(&a_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
           const uint32_t fb = sm100::smem_u32(&a_full[s]);
@@ -191,7 +199,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     int s = 0, sa = 0;
     uint64_t wd = wdesc0, ad = adesc0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const Item w = decode_item(g, item);
+      const Item w = decode_item<MODE>(g, item);
       const int kb0 = w.kb0, kb1 = w.kb1;
       uint32_t acc = 0u;                 // the watcher's first release of an item also says that the accumulator is free
       for (int kb = kb0; kb < kb1; ++kb) {
@@ -233,7 +241,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // longer holds, so from then on the watcher meets the MMA warp at every barrier instead.
     int s = 0, sa = 0; uint32_t ph = 0, pha = 0, it = 0; bool failed = false;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-      const Item w = decode_item(g, item);
+      const Item w = decode_item<MODE>(g, item);
       if (!failed) {
         bool ok = true;
         if (lane == 0) ok = sm100::mbar_wait(sm100::smem_u32(&tmem_empty_bar), (it & 1u) ^ 1u, abortp);
@@ -281,7 +289,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
     };
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-      const Item w = decode_item(g, item);
+      const Item w = decode_item<MODE>(g, item);
       const int split = w.split, tile = w.tile, rb = w.rb;
       if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
       sm100::tc_fence_after();

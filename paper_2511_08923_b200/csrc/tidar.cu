@@ -37,6 +37,8 @@ struct tidar_ctx {
   const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<const bf16 *> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   // geometry
+  int R_head = 0;                  // rows of a pass that can get logits (the rows of a decode step)
+  int last_hidden_off = 0;         // first row of the last pass that the read-back calls address
   int R_cap = 0, T_max = 0, pages_per_seq = 0, n_pages = 0, n_qkv = 0, S_max = 4, lm_chunk = 0;
   size_t pool_stride = 0;    // elements in one layer's K (or V) pool
   size_t partial_stride = 0; // elements between split-K partial slabs
@@ -134,6 +136,7 @@ int validate(const tidar_config &c, std::string &why) {
   if (!(c.beta >= 0.0f && c.beta <= 1.0f)) return bad("beta must be in [0, 1]");
   if (c.temperature != 0.0f) return bad("only greedy decoding (temperature 0) is implemented");
   if (c.impl != 0 && c.impl != 1) return bad("impl must be 0 (tensor-core kernels) or 1 (replay kernels)");
+  if (c.prefill_rows < 0 || c.prefill_rows > (1 << 16)) return bad("prefill_rows must be in [0, 65536]");
   if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return bad("rms_eps > 0 and rope_theta > 1 required");
   return TIDAR_OK;
 }
@@ -142,7 +145,8 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   const tidar_config &c = x.cfg;
   x.T_max = c.k_max * (c.k_max + 1);
   // rows of a pass: the step's slots, plus one mixed row per verified position when beta < 1
-  x.R_cap = (int)align_up((size_t)std::max(c.max_batch * (x.T_max + (c.beta < 1.0f ? c.k_max : 0)), 256), 16);
+  x.R_head = (int)align_up((size_t)std::max(c.max_batch * (x.T_max + (c.beta < 1.0f ? c.k_max : 0)), 256), 16);
+  x.R_cap = std::max(x.R_head, (int)align_up((size_t)std::max(c.prefill_rows, 0), 16));
   x.pages_per_seq = (c.max_seq_len + c.page_size - 1) / c.page_size;
   x.n_pages = x.pages_per_seq * c.max_batch;
   x.n_qkv = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
@@ -193,7 +197,7 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.dbg_kv = cv.take<bf16>((size_t)2 * 256 * c.n_kv_heads * c.head_dim);
   if (c.debug & 1) {
     x.dbg_hidden = cv.take<float>((size_t)(c.n_layers + 1) * R * c.d_model);
-    x.dbg_logits = cv.take<float>(R * (size_t)c.vocab);
+    x.dbg_logits = cv.take<float>((size_t)x.R_head * (size_t)c.vocab);
   }
   *bytes = align_up(cv.off, 256);
 }
@@ -485,7 +489,9 @@ void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t strid
 // Extra LM-head input rows that mix two final-normed rows each (beta < 1; see mix_rows_kernel).
 struct MixRows { int n = 0, k = 1, a0 = 0, a_seq = 0, a_j = 0, b0 = 0, b_seq = 0, b_j = 0; };
 
-int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int key_tiles_hint, const MixRows &mix = MixRows()) {
+// head_row0: the LM head (with_head) runs on rows [head_row0, R) only, followed by the mixed rows; the
+// argmax ids and the logits dump are indexed from head_row0.
+int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int key_tiles_hint, const MixRows &mix = MixRows(), int head_row0 = 0) {
   const tidar_config &cf = c->cfg;
   const int d = cf.d_model, hd = cf.head_dim, Hq = cf.n_q_heads, Hkv = cf.n_kv_heads;
   const KvGeom g = geom(c);
@@ -542,18 +548,21 @@ if (tc && c->slab_bf16)
     launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, R, lm.tl);
     R += mix.n;
   }
+  const bf16 *Ah = c->A + (size_t)head_row0 * d;           // first row of the LM head's input
+  const int Rh = R - head_row0;
+  if (with_head && Rh > c->R_head) return fail(c, TIDAR_ECAPACITY, "%d rows for the LM head exceed the context's %d", Rh, c->R_head);
   if (with_head && tc) {
     const int G = c->n_sms * 4;          // upper bound of (CTAs of the LM-head kernel) x 4 lane quadrants
-    CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * R * sizeof(int32_t), c->stream));
-    if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, c->A, RA, c->tm_lm, R, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
+    CUDA_TRY(c, cudaMemsetAsync(c->cand_idx, 0xff, (size_t)G * Rh * sizeof(int32_t), c->stream));
+    if ((rc = gemm_tc_launch(c, gemm_tc::MODE_ARGMAX, Ah, RA - head_row0, c->tm_lm, Rh, cf.vocab, d, TIDAR_TC_LMHEAD, nullptr, nullptr))) return rc;
     Launch ll(c, TIDAR_TC_LMHEAD);
-    launch_after(argmax_merge_kernel, (R * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, R, c->d_arg_val, c->d_arg_idx, ll.tl);
+    launch_after(argmax_merge_kernel, (Rh * 32 + 255) / 256, 256, 0, c->stream, c->cand_val, c->cand_idx, G, Rh, c->d_arg_val, c->d_arg_idx, ll.tl);
   } else if (with_head) {
     for (int v0 = 0; v0 < cf.vocab; v0 += c->lm_chunk) {
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
-      if ((rc = gemm_partials(c, c->A, RA, c->lm_head + (size_t)v0 * d, nullptr, R, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD))) return rc;
+      if ((rc = gemm_partials(c, Ah, RA - head_row0, c->lm_head + (size_t)v0 * d, nullptr, Rh, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD))) return rc;
       Launch ll(c, TIDAR_TC_LMHEAD);
-      argmax_chunk_kernel<<<R, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab);
+      argmax_chunk_kernel<<<Rh, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab);
     }
   }
   CUDA_TRY(c, cudaGetLastError());
@@ -756,6 +765,7 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   c->pending_k = k;
   c->pending_seqs.assign(seqs, seqs + n_seqs);
   c->pending = true;
+  c->last_hidden_off = 0;
   c->last_rows = R + ((cf.beta < 1.0f && !ar) ? n_seqs * k : 0); c->last_first_pos = -1;      // the mixed rows follow the slots
   // the host tracks lengths without reading the device when L is forced
   return TIDAR_OK;
@@ -880,12 +890,15 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
     MixRows mix;
     const int rlp = n_prompt - 1 - row0;               // the last prompt row inside this chunk
     if (last && cf.beta < 1.0f) { mix.n = 1; mix.k = 1; mix.a0 = rlp; mix.b0 = rlp + 1; }
-    if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64, mix)) return rc;
+    // logits are needed for the last prompt row and the k mask rows only; the LM head runs on the
+    // trailing rows of the last chunk, as many as a decode step has (all of them for a short prompt)
+    const int head_row0 = last ? std::max(0, rows + mix.n - c->R_head) : 0;
+    if (int rc = forward_rows(c, rows, last, rows, (row0 + rows / 2 + 63) / 64, mix, head_row0)) return rc;
     if (last) {
       Launch l(c, TIDAR_TC_VERIFY);
-      prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, rlp, mix.n ? rows : rlp, k, cf.k_max, seq, n_prompt, c->d_block,
-                                                     c->d_blk_len, c->d_seq_len, c->d_out);
-      c->last_rows = rows; c->last_first_pos = row0;
+      prefill_finish_kernel<<<1, 32, 0, c->stream>>>(c->d_arg_idx, rlp - head_row0, (mix.n ? rows : rlp) - head_row0, k, cf.k_max, seq, n_prompt,
+                                                     c->d_block, c->d_blk_len, c->d_seq_len, c->d_out);
+      c->last_rows = rows - head_row0; c->last_first_pos = row0 + head_row0; c->last_hidden_off = head_row0;
     }
     row0 += rows;
   }
@@ -1048,7 +1061,8 @@ int tidar_debug_get_hidden(tidar_ctx *c, int32_t layer, int32_t row0, int32_t n,
   if (layer < 0 || layer > c->cfg.n_layers) return fail(c, TIDAR_EINVAL, "layer out of range");
   if (int rc = check_rows(c, row0, n)) return rc;
   const size_t d = c->cfg.d_model;
-  CUDA_TRY(c, cudaMemcpyAsync(out, c->dbg_hidden + ((size_t)layer * c->R_cap + row0) * d, (size_t)n * d * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(out, c->dbg_hidden + ((size_t)layer * c->R_cap + c->last_hidden_off + row0) * d, (size_t)n * d * sizeof(float),
+                              cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return TIDAR_OK;
 }

@@ -34,7 +34,7 @@ def test_library_builds_and_exports_every_declared_symbol():
 def _cfg(**over):
     base = dict(n_layers=2, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, d_ffn=704, vocab=1024, tie_lm_head=1,
                 rms_eps=1e-6, rope_theta=1e4, mask_token_id=1023, k_max=4, max_batch=1, max_seq_len=256, page_size=64,
-                beta=1.0, temperature=0.0, sample_seed=0, debug=0, impl=1)
+                beta=1.0, temperature=0.0, sample_seed=0, debug=0, impl=1, prefill_rows=0)
     base.update(over)
     return binding.tidar_config(**base)
 

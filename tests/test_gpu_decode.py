@@ -14,12 +14,12 @@ pytestmark = pytest.mark.gpu
 IMPLS = [0, 1]
 
 
-def _gpu(sh, wt, impl, k_max=None, debug=1, max_batch=1, max_seq_len=512):
+def _gpu(sh, wt, impl, k_max=None, debug=1, max_batch=1, max_seq_len=512, prefill_rows=0):
     """A context whose arena is followed by 64 KiB of sentinel bytes; _close() checks them."""
     from paper_2511_08923_b200 import Tidar, pack_weights
     packed = pack_weights(wt, "cuda:0")
     return Tidar(sh, packed, k_max=k_max or sh.k, max_batch=max_batch, max_seq_len=max_seq_len, debug=debug, impl=impl,
-                 guard_bytes=64 * 1024)
+                 guard_bytes=64 * 1024, prefill_rows=prefill_rows)
 
 
 def _close(t):
@@ -381,3 +381,45 @@ def test_device_timeout_status_is_reported_and_sequences_released(tiny, impl):
     assert e.value.code == -5
     t.sync()                                        # the word was cleared by the report
     _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_long_first_pass_in_one_chunk(tiny, impl):
+    """prefill_rows: a 700-token prompt encoded in ONE pass of 704 rows (three row blocks of the
+    projections, weight tiles shared between them; the LM head on the trailing rows only) against the
+    oracle, and against the same prompt encoded in the default chunks of 256 rows."""
+    from paper_2511_08923_b200 import bf16_bits_to_f32
+    sh, wt, cfg, w, _ = tiny
+    k = sh.k
+    prompt = prompt_ids(sh, 700, seed=9)
+    n = len(prompt)
+    st, c, fo = O.prefill(cfg, w, prompt, k, return_forward=True)
+    outs = []
+    for rows in (768, 0):
+        t = _gpu(sh, wt, impl, max_seq_len=1024, prefill_rows=rows)
+        first = t.prefill(0, prompt, k)
+        n_rows, row0 = t.last_rows()
+        assert row0 + n_rows == n + k and row0 <= n - 1
+        if rows:
+            assert n_rows == 256 and row0 == n + k - 256          # logits for the trailing rows of the single chunk
+        lg = t.logits(0, n_rows)
+        assert np.abs(lg - fo.logits[row0:]).max() <= TOL_LOGITS
+        for l in range(cfg.n_layers + 1):
+            assert np.abs(t.hidden(l, 0, n_rows) - fo.hidden[l][row0:]).max() <= TOL_LOGITS
+        ids = t.argmax(0, n_rows)
+        np.testing.assert_array_equal(ids, lg.argmax(-1))
+        assert first == int(lg[n - 1 - row0].argmax())
+        assert t.get_block(0, k) == [first] + [int(x) for x in lg[n + 1 - row0:n + k - row0].argmax(-1)]
+        kv = []
+        for l in range(cfg.n_layers):
+            kk, vv = t.kv(0, l, 0, n)
+            assert np.abs(bf16_bits_to_f32(kk) - st.k_cache[l]).max() <= TOL_LOGITS
+            assert np.abs(bf16_bits_to_f32(vv) - st.v_cache[l]).max() <= TOL_LOGITS
+            kv.append((kk, vv))
+        toks, L = t.step([0], forced=[2])
+        outs.append((first, kv, toks, t.get_block(0, k)))
+        _close(t)
+    # layer 0's cache does not depend on how the prompt was cut into passes
+    np.testing.assert_array_equal(outs[0][1][0][0], outs[1][1][0][0]); np.testing.assert_array_equal(outs[0][1][0][1], outs[1][1][0][1])
+    if top1_margin(fo.logits[n - 1]) > MARGIN:
+        assert outs[0][0] == outs[1][0] == c
