@@ -96,11 +96,17 @@ typedef struct {
  *                  that one tile of output rows holds matching gate/up pairs)
  *   w_down[l]    : [d_model][d_ffn]
  *   embed, lm_head : [vocab][d_model];  *_norm : [d_model] bf16 gains
- * The six per-layer arrays are HOST arrays of n_layers device pointers.            */
+ * The per-layer arrays are HOST arrays of n_layers device pointers.
+ * Optional (NULL = absent; the paper starts from Qwen2.5 and Qwen3 decoders, Section 4.1,
+ * whose attention blocks differ in these two details):
+ *   bqkv[l]   : [(n_q_heads + 2*n_kv_heads)*head_dim] bf16, bias added to the QKV projection
+ *   q_norm[l], k_norm[l] : [head_dim] bf16 gains of an RMSNorm (rms_eps) over the dimensions of
+ *               every Q head / K head, applied before RoPE; given together or not at all   */
 typedef struct {
   const void *embed, *lm_head, *final_norm;
   const void *const *attn_norm, *const *wqkv, *const *wo;
   const void *const *ffn_norm, *const *w_gate_up, *const *w_down;
+  const void *const *bqkv, *const *q_norm, *const *k_norm;
 } tidar_weights;
 
 /* Bytes of device memory the context needs for cfg (KV pages, activations, scratch).

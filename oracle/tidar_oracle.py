@@ -33,9 +33,12 @@ mask slot (b, i) sits at position ``n + b + 1 + i``; block b sees causal slots
 causal slot is the token already settled by the previous pass, so acceptance
 lengths run over 1..k; ties in argmax go to the lowest index.
 
-Model family (the paper continues pre-training from Qwen-type decoders): pre-norm
-decoder, RMSNorm, grouped-query attention with rotate-half RoPE, SwiGLU FFN,
-no biases.
+Model family (the paper continues pre-training from Qwen2.5 and Qwen3 decoders,
+Section 4.1): pre-norm decoder, RMSNorm, grouped-query attention with rotate-half
+RoPE, SwiGLU FFN.  The two checkpoint families differ in two details, both optional
+here and absent from the benchmark configurations: biases on the Q/K/V projections
+(layer keys "bq", "bk", "bv") and an RMSNorm over each head's dimensions of Q and K
+before RoPE (layer keys "q_norm", "k_norm").
 
 parity pins: see tests/test_oracle_*.py.  Numeric values of hidden states and
 logits have no printed example in the paper; they are pinned by a brute-force
@@ -250,9 +253,13 @@ def forward(cfg: OracleConfig, w: dict, ids: np.ndarray, pos: np.ndarray, mask: 
     for l, L in enumerate(w["layers"]):
         hidden.append(x.copy())
         a = _stored(cfg, rmsnorm(x, L["attn_norm"], cfg.rms_eps))
-        q = (a @ L["wq"].T).reshape(R, Hq, hd)
-        kk = (a @ L["wk"].T).reshape(R, Hkv, hd)
-        vv = _stored(cfg, (a @ L["wv"].T).reshape(R, Hkv, hd))
+        q, kk, vv = a @ L["wq"].T, a @ L["wk"].T, a @ L["wv"].T
+        if "bq" in L:                                   # projection biases (one checkpoint family)
+            q, kk, vv = q + L["bq"], kk + L["bk"], vv + L["bv"]
+        q, kk, vv = q.reshape(R, Hq, hd), kk.reshape(R, Hkv, hd), vv.reshape(R, Hkv, hd)
+        if "q_norm" in L:                               # per-head RMSNorm of Q and K before RoPE (the other family)
+            q, kk = rmsnorm(q, L["q_norm"], cfg.rms_eps), rmsnorm(kk, L["k_norm"], cfg.rms_eps)
+        vv = _stored(cfg, vv)
         q = _stored(cfg, rope(q, pos, cfg.rope_theta))
         kk = _stored(cfg, rope(kk, pos, cfg.rope_theta))
         k_new.append(kk); v_new.append(vv)

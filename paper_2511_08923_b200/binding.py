@@ -40,7 +40,8 @@ class tidar_config(C.Structure):
 
 class tidar_weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] + \
-               [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")]
+               [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down",
+                                                     "bqkv", "q_norm", "k_norm")]
 
 
 _lib = None
@@ -118,11 +119,16 @@ def pack_weights(w: dict, device) -> dict:
     out["layers"] = []
     for L in w["layers"]:
         gu = torch.stack([L["w_gate"], L["w_up"]], dim=1).reshape(2 * L["w_gate"].shape[0], L["w_gate"].shape[1])
-        out["layers"].append({
+        lay = {
             "attn_norm": dev(L["attn_norm"]), "ffn_norm": dev(L["ffn_norm"]),
             "wqkv": dev(torch.cat([L["wq"], L["wk"], L["wv"]], dim=0)),
             "wo": dev(L["wo"]), "w_gate_up": dev(gu), "w_down": dev(L["w_down"]),
-        })
+        }
+        if "bq" in L:
+            lay["bqkv"] = dev(torch.cat([L["bq"], L["bk"], L["bv"]], dim=0))
+        if "q_norm" in L:
+            lay["q_norm"], lay["k_norm"] = dev(L["q_norm"]), dev(L["k_norm"])
+        out["layers"].append(lay)
     return out
 
 
@@ -160,6 +166,9 @@ class Tidar:
         arrs = {}
         for name in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
             arrs[name] = (C.c_void_p * nl)(*[L[name].data_ptr() for L in packed["layers"]])
+        for name in ("bqkv", "q_norm", "k_norm"):          # optional: present in every layer or in none
+            if nl and name in packed["layers"][0]:
+                arrs[name] = (C.c_void_p * nl)(*[L[name].data_ptr() for L in packed["layers"]])
         self._arrs = arrs
         wts = tidar_weights(embed=packed["embed"].data_ptr(), lm_head=packed["lm_head"].data_ptr(),
                             final_norm=packed["final_norm"].data_ptr(),

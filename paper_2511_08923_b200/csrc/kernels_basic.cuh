@@ -175,13 +175,17 @@ rmsnorm_reduce_kernel(float *__restrict__ X, const SLAB *__restrict__ partials, 
 // rotated, V heads copied; both go to the paged cache at the row's cache position
 // (causal slots: kept if accepted, evicted otherwise; paper Section 3.3) or to the
 // step-local scratch (mask slots, never cached).  Grid (rows, unit chunks of 256).
+// Optional, for checkpoints of the decoder families the paper starts from (Section 4.1):
+// bias [(Hq+2Hkv)*hd] added to the projection; qn / kn [hd]: RMSNorm over each Q / K head's
+// dimensions before the rotation (the hd/8 threads of a head reduce with shuffles).
 // ---------------------------------------------------------------------------
 template <typename SLAB>
 __global__ void __launch_bounds__(256)
 rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, int Hq, int Hkv, int hd,
                RowMeta m, const float *__restrict__ cs, const float *__restrict__ sn, KvGeom g,
                bf16 *__restrict__ Q, bf16 *__restrict__ Kpool, bf16 *__restrict__ Vpool,
-               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc, TlSlot tl) {
+               bf16 *__restrict__ Kloc, bf16 *__restrict__ Vloc,
+               const bf16 *__restrict__ bias, const bf16 *__restrict__ qn, const bf16 *__restrict__ kn, float eps, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
@@ -200,6 +204,28 @@ rope_kv_kernel(const SLAB *__restrict__ partials, int S, size_t partial_stride, 
       const float4 b = load4<SLAB>(partials + s * partial_stride + base + half);
       x1.x += a.x; x1.y += a.y; x1.z += a.z; x1.w += a.w;
       x2.x += b.x; x2.y += b.y; x2.z += b.z; x2.w += b.w;
+    }
+    if (bias) {
+      const uint2 b1 = *reinterpret_cast<const uint2 *>(bias + (size_t)h * hd + i), b2 = *reinterpret_cast<const uint2 *>(bias + (size_t)h * hd + i + half);
+      const float2 p0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&b1.x)), p1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&b1.y));
+      const float2 q0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&b2.x)), q1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&b2.y));
+      x1.x += p0.x; x1.y += p0.y; x1.z += p1.x; x1.w += p1.y;
+      x2.x += q0.x; x2.y += q0.y; x2.z += q1.x; x2.w += q1.y;
+    }
+    const bf16 *hn = h < Hq ? qn : (h < Hq + Hkv ? kn : nullptr);
+    if (hn) {
+      // the upr = hd/8 threads of this head are consecutive lanes of one warp (upr is 8 or 16 and
+      // divides the unit index), and all of them are here: the loop bound is a multiple of upr
+      float ss = x1.x * x1.x + x1.y * x1.y + x1.z * x1.z + x1.w * x1.w + x2.x * x2.x + x2.y * x2.y + x2.z * x2.z + x2.w * x2.w;
+      const int lane = threadIdx.x & 31;
+      const unsigned gmask = (upr >= 32 ? 0xffffffffu : ((1u << upr) - 1u)) << (lane & ~(upr - 1));
+      for (int o = upr >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(gmask, ss, o);
+      const float inv = rsqrtf(ss / (float)hd + eps);
+      const uint2 g1 = *reinterpret_cast<const uint2 *>(hn + i), g2 = *reinterpret_cast<const uint2 *>(hn + i + half);
+      const float2 p0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&g1.x)), p1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&g1.y));
+      const float2 q0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&g2.x)), q1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&g2.y));
+      x1.x *= inv * p0.x; x1.y *= inv * p0.y; x1.z *= inv * p1.x; x1.w *= inv * p1.y;
+      x2.x *= inv * q0.x; x2.y *= inv * q0.y; x2.z *= inv * q1.x; x2.w *= inv * q1.y;
     }
     bf16 *dst;
     bool rotate = true;

@@ -36,6 +36,7 @@ struct tidar_ctx {
   // borrowed weights
   const bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<const bf16 *> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
+  std::vector<const bf16 *> bqkv, q_norm, k_norm;      // optional (empty = absent)
   // geometry
   int R_head = 0;                  // rows of a pass that can get logits (the rows of a decode step)
   int last_hidden_off = 0;         // first row of the last pass that the read-back calls address
@@ -514,12 +515,14 @@ int forward_rows(tidar_ctx *c, int R, bool with_head, int rows_per_group, int ke
     {
       Launch ll(c, TIDAR_TC_ROPE);
       const int rope_chunks = ((Hq + 2 * Hkv) * (hd / 8) + 255) / 256;
+      const bf16 *bias_l = c->bqkv.empty() ? nullptr : c->bqkv[l], *qn_l = c->q_norm.empty() ? nullptr : c->q_norm[l],
+                 *kn_l = c->k_norm.empty() ? nullptr : c->k_norm[l];
 if (tc && c->slab_bf16)
         launch_after(rope_kv_kernel<bf16>, dim3(R, rope_chunks), 256, 0, c->stream, (const bf16 *)c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
-                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, ll.tl);
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, bias_l, qn_l, kn_l, cf.rms_eps, ll.tl);
       else
         launch_after(rope_kv_kernel<float>, dim3(R, rope_chunks), 256, 0, c->stream, c->partials, S, stride, Hq, Hkv, hd, c->meta, c->rope_cos,
-                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, ll.tl);
+                                                                      c->rope_sin, g, c->Q, Kp, Vp, c->Kloc, c->Vloc, bias_l, qn_l, kn_l, cf.rms_eps, ll.tl);
     }
     if (tc) {
       AttnMaps am{&c->tm_q, &c->tm_kv, &c->tm_kv, &c->tm_kloc, &c->tm_vloc, (2 * l) * c->n_pages, (2 * l + 1) * c->n_pages};
@@ -836,6 +839,14 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
     c->attn_norm.push_back((const bf16 *)w->attn_norm[l]); c->wqkv.push_back((const bf16 *)w->wqkv[l]);
     c->wo.push_back((const bf16 *)w->wo[l]); c->ffn_norm.push_back((const bf16 *)w->ffn_norm[l]);
     c->wgu.push_back((const bf16 *)w->w_gate_up[l]); c->wdown.push_back((const bf16 *)w->w_down[l]);
+  }
+  if ((w->q_norm != nullptr) != (w->k_norm != nullptr)) { delete c; return fail(nullptr, TIDAR_EINVAL, "q_norm and k_norm come together or not at all"); }
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (w->bqkv) { if (!w->bqkv[l]) { delete c; return fail(nullptr, TIDAR_EINVAL, "null bqkv pointer in layer %d", l); } c->bqkv.push_back((const bf16 *)w->bqkv[l]); }
+    if (w->q_norm) {
+      if (!w->q_norm[l] || !w->k_norm[l]) { delete c; return fail(nullptr, TIDAR_EINVAL, "null q_norm / k_norm pointer in layer %d", l); }
+      c->q_norm.push_back((const bf16 *)w->q_norm[l]); c->k_norm.push_back((const bf16 *)w->k_norm[l]);
+    }
   }
   if (cfg->impl == 0) {
     if (int rc = init_tensor_core_path(c)) { std::string m = c->err; delete c; return fail(nullptr, rc, "%s", m.c_str()); }

@@ -7,7 +7,7 @@ import pytest
 import torch  # noqa: F401
 
 from oracle import tidar_oracle as O
-from tests.helpers import MARGIN, TOL_LOGITS, make_model, oracle_cfg, prompt_ids, top1_margin
+from tests.helpers import MARGIN, TOL_LOGITS, check_rows, make_model, oracle_cfg, prompt_ids, top1_margin
 
 pytestmark = pytest.mark.gpu
 
@@ -160,4 +160,42 @@ def test_beta_mixed_verification(tiny, impl, beta):
             assert L[0] == so.L and toks[0] == so.emitted
         elif L[0] != so.L:
             break
+    _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("family,hd", [("bias", 64), ("qk_norm", 64), ("bias", 128), ("qk_norm", 128)])
+def test_projection_bias_and_per_head_qk_norm(impl, family, hd):
+    """The two attention-block details in which the decoder families the paper starts from differ
+    (Section 4.1): biases on Q/K/V, or an RMSNorm over each Q / K head before RoPE.  First pass and
+    teacher-forced steps against the oracle, for both head widths the kernels support."""
+    from paper_2511_08923_b200 import bf16_bits_to_f32
+    from tidar_synth import CONFIGS, gen_model_weights
+    over = dict(head_dim=hd, n_q_heads=4, n_kv_heads=2, d_model=256) if hd == 64 else dict(head_dim=hd, n_q_heads=6, n_kv_heads=2, d_model=512, d_ffn=768)
+    sh = replace(CONFIGS["tiny"], name=f"{family}{hd}", tie_lm_head=False, qkv_bias=family == "bias", qk_norm=family == "qk_norm", **over)
+    wt = gen_model_weights(sh)
+    cfg, w = oracle_cfg(sh), O.weights_to_f64(wt)
+    prompt = prompt_ids(sh, 70)
+    k, n = sh.k, 70
+    t = _gpu(sh, wt, impl, k_max=k, debug=1)
+    t.prefill(0, prompt, k)
+    st, c, fo = O.prefill(cfg, w, prompt, k, return_forward=True)
+    assert np.abs(t.logits(0, n + k) - fo.logits).max() <= TOL_LOGITS
+    for l in range(cfg.n_layers):                   # normed K reaches |x| ~ 5, where one bf16 ulp is 0.03: bound by the row's scale
+        kk, vv = t.kv(0, l, 0, n)
+        check_rows(bf16_bits_to_f32(kk).reshape(n, -1), st.k_cache[l].reshape(n, -1), f"K({l})")
+        check_rows(bf16_bits_to_f32(vv).reshape(n, -1), st.v_cache[l].reshape(n, -1), f"V({l})")
+    # the same weights without the extra tensors give clearly different logits: the option is live on the GPU
+    plain = {**wt, "layers": [{a: b for a, b in L.items() if a not in ("bq", "bk", "bv", "q_norm", "k_norm")} for L in wt["layers"]]}
+    t0 = _gpu(sh, plain, impl, k_max=k, debug=1)
+    t0.prefill(0, prompt, k)
+    assert np.abs(t0.logits(0, n + k) - fo.logits).max() > 10 * TOL_LOGITS
+    _close(t0)
+    for s in range(2):
+        t.set_block(0, st.block)
+        so = O.step(cfg, w, st, forced=2)
+        toks, L = t.step([0], forced=[2])
+        assert np.abs(t.logits(0, k * (k + 1)) - so.fwd.logits).max() <= TOL_LOGITS
+        if (top1_margin(so.fwd.logits[:k]) > MARGIN).all():
+            assert toks[0] == so.emitted
     _close(t)

@@ -198,3 +198,44 @@ def test_bf16_storage_mode_rounds_only_what_is_stored():
     d = np.abs(a.logits - b.logits).max()
     assert 1e-5 < d < 3e-2, d
     np.testing.assert_array_equal(a.hidden[0], b.hidden[0])        # the embedding rows are not an activation store
+
+
+# ---- optional projection biases and per-head Q/K norm: pinned against library decoders that have them
+def _hf_state(wt, extra):
+    sd = {"model.embed_tokens.weight": wt["embed"], "model.norm.weight": wt["final_norm"], "lm_head.weight": wt["lm_head"]}
+    names = {"wq": "self_attn.q_proj.weight", "wk": "self_attn.k_proj.weight", "wv": "self_attn.v_proj.weight", "wo": "self_attn.o_proj.weight",
+             "w_gate": "mlp.gate_proj.weight", "w_up": "mlp.up_proj.weight", "w_down": "mlp.down_proj.weight",
+             "attn_norm": "input_layernorm.weight", "ffn_norm": "post_attention_layernorm.weight", **extra}
+    for l, L in enumerate(wt["layers"]):
+        for k_, v_ in names.items():
+            sd[f"model.layers.{l}.{v_}"] = L[k_]
+    return {k_: v_.double() for k_, v_ in sd.items()}
+
+
+@pytest.mark.parametrize("family", ["qwen2_bias", "qwen3_qk_norm"])
+def test_causal_forward_with_bias_or_qk_norm_matches_transformers(family):
+    tf = pytest.importorskip("transformers")
+    from dataclasses import replace
+    sh = replace(CONFIGS["tiny"], tie_lm_head=False, qkv_bias=family == "qwen2_bias", qk_norm=family == "qwen3_qk_norm")
+    wt = gen_model_weights(sh)
+    cfg = _cfg(sh)
+    w = O.weights_to_f64(wt)
+    ids = gen_token_ids(4, tensor_id("prompt"), 19, sh.vocab - 1).numpy().astype(np.int64)
+    fo = O.causal_forward(cfg, w, ids)
+    common = dict(vocab_size=sh.vocab, hidden_size=sh.d_model, intermediate_size=sh.d_ffn, num_hidden_layers=sh.n_layers,
+                  num_attention_heads=sh.n_q_heads, num_key_value_heads=sh.n_kv_heads, rms_norm_eps=sh.rms_eps, rope_theta=sh.rope_theta,
+                  tie_word_embeddings=False, max_position_embeddings=512, attn_implementation="eager", use_sliding_window=False)
+    if family == "qwen2_bias":
+        m = tf.Qwen2ForCausalLM(tf.Qwen2Config(**common)).double().eval()
+        extra = {"bq": "self_attn.q_proj.bias", "bk": "self_attn.k_proj.bias", "bv": "self_attn.v_proj.bias"}
+    else:
+        m = tf.Qwen3ForCausalLM(tf.Qwen3Config(head_dim=sh.head_dim, attention_bias=False, **common)).double().eval()
+        extra = {"q_norm": "self_attn.q_norm.weight", "k_norm": "self_attn.k_norm.weight"}
+    missing = m.load_state_dict(_hf_state(wt, extra), strict=False)
+    assert not [x for x in missing.missing_keys if "rotary" not in x] and not missing.unexpected_keys
+    with torch.no_grad():
+        ref = m(torch.from_numpy(ids)[None]).logits[0].numpy()
+    np.testing.assert_allclose(fo.logits, ref, rtol=0, atol=2e-6)
+    # and the option does something: the same weights without it give different logits
+    plain = {**w, "layers": [{k_: v_ for k_, v_ in L.items() if k_ not in extra} for L in w["layers"]]}
+    assert np.abs(O.causal_forward(cfg, plain, ids).logits - fo.logits).max() > 1e-3

@@ -108,6 +108,7 @@ _KINDS = {
     "embed": 1, "lm_head": 2, "final_norm": 3,
     "attn_norm": 10, "wq": 11, "wk": 12, "wv": 13, "wo": 14,
     "ffn_norm": 15, "w_gate": 16, "w_up": 17, "w_down": 18,
+    "bq": 19, "bk": 20, "bv": 21, "q_norm": 22, "k_norm": 23,
     "prompt": 30, "drafts": 31, "q": 40, "k": 41, "v": 42, "perm": 43,
 }
 TID_SCHEDULE = 50 << 12
@@ -135,6 +136,8 @@ class ModelShape:
     rms_eps: float = 1e-6
     seed: int = 0
     init_std: float = 0.02
+    qkv_bias: bool = False       # biases on the Q/K/V projections
+    qk_norm: bool = False        # RMSNorm over each head's dimensions of Q and K before RoPE
     # workload
     prompt_len: int = 64
     k: int = 4
@@ -193,8 +196,19 @@ def gen_model_weights(shape: ModelShape, device="cpu", layers=None, with_head: b
              "final_norm": gain("final_norm", 0)}
         w["lm_head"] = w["embed"] if shape.tie_lm_head else mat("lm_head", 0, shape.vocab, d)
     w["layers"] = []
+    def vec(kind, layer, n, scale, offset):
+        g = gen_normal_bf16(s, tensor_id(kind, layer), n, scale, device).to(torch.float32)
+        return (offset + g).to(torch.bfloat16)
+
     for l in (range(shape.n_layers) if layers is None else layers):
+        extra = {}
+        if shape.qkv_bias:
+            extra.update(bq=vec("bq", l, shape.n_q_heads * hd, 0.1, 0.0), bk=vec("bk", l, shape.n_kv_heads * hd, 0.1, 0.0),
+                         bv=vec("bv", l, shape.n_kv_heads * hd, 0.1, 0.0))
+        if shape.qk_norm:
+            extra.update(q_norm=vec("q_norm", l, hd, 0.1, 1.0), k_norm=vec("k_norm", l, hd, 0.1, 1.0))
         w["layers"].append({
+            **extra,
             "index": l,
             "attn_norm": gain("attn_norm", l),
             "wq": mat("wq", l, shape.n_q_heads * hd, d),
