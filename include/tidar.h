@@ -65,8 +65,18 @@ typedef struct {
                                1.0 (verification by the autoregressive prediction alone) is
                                the hot path and makes greedy TiDAR equal greedy AR decoding;
                                below 1 every verified position costs one more LM-head row  */
-  float   temperature;      /* 0 = greedy; only greedy is implemented                      */
-  uint64_t sample_seed;     /* reserved for seeded sampling                                */
+  float   temperature;      /* 0 = greedy (the hot path).  > 0: every prediction (verified
+                               targets and drafts alike) is a draw from softmax(logits /
+                               temperature) by the Gumbel-max rule, and a draft is accepted
+                               iff it equals the drawn target (paper Section 3.2 read as
+                               token match).  The noise of a draw is a pure function of
+                               (sample_seed, sequence slot, predicted position, token id):
+                               SplitMix64's mix of (seed, slot, position) gives a 32-bit key,
+                               MurmurHash3's fmix32(key + id * 0x9E3779B9) the 24 uniform bits
+                               of -ln(-ln u).  Draws therefore do not depend on how positions
+                               fall into passes, and with beta = 1 the emitted sequence equals
+                               one-token-per-pass sampling with the same rule                */
+  uint64_t sample_seed;     /* seed of the sampling noise                                  */
   int32_t debug;            /* bit 0: keep per-layer hidden states and full logits of the
                                last pass for the tidar_debug_get_* calls (costs memory:
                                rows*vocab*4 bytes); bit 1: overwrite evicted KV slots with

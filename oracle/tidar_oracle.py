@@ -76,6 +76,12 @@ class OracleConfig:
     # SwiGLU output) are rounded to bfloat16 where they are stored; the paper trains and runs in
     # "standard BFloat 16" (Section 4.1).  All arithmetic stays float64 in both modes.
     act_dtype: str = "f64"
+    # temperature 0: every prediction is the argmax (the hot path).  temperature > 0: every prediction is
+    # a draw from softmax(logits / temperature), taken with noise that depends only on (sample_seed,
+    # seq, predicted position, token id): see choose_tokens.
+    temperature: float = 0.0
+    sample_seed: int = 0
+    seq: int = 0
 
 
 @dataclass
@@ -285,6 +291,65 @@ def argmax_lowest(x: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------
+# seeded sampling  (Section 3.2: drafts are sampled and then checked against the autoregressive
+# prediction; read as token match, so "sampling" means: every prediction is a draw)
+# ----------------------------------------------------------------------------
+_M64 = (1 << 64) - 1
+
+
+def mix64(z: int) -> int:
+    """The output function of SplitMix64 (Steele, Lea, Flood 2014): a bijection of 64-bit words."""
+    z &= _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def fmix32(h: np.ndarray) -> np.ndarray:
+    """The 32-bit finaliser of MurmurHash3 (Appleby), element-wise on uint32."""
+    h = h.astype(np.uint32)
+    h ^= h >> np.uint32(16)
+    h = (h * np.uint32(0x85EBCA6B)).astype(np.uint32)
+    h ^= h >> np.uint32(13)
+    h = (h * np.uint32(0xC2B2AE35)).astype(np.uint32)
+    h ^= h >> np.uint32(16)
+    return h
+
+
+def position_key(seed: int, seq: int, pos: int) -> int:
+    """32-bit key of one predicted position of one sequence: the top half of
+    mix64(mix64(seed + golden ratio) ^ (seq << 32 | pos))."""
+    return mix64(mix64(seed + 0x9E3779B97F4A7C15) ^ (((seq & 0xFFFFFFFF) << 32) | (pos & 0xFFFFFFFF))) >> 32
+
+
+def gumbel_noise(seed: int, seq: int, pos: int, vocab: int) -> np.ndarray:
+    """Standard Gumbel noise for every token id of one predicted position: u = (top 24 bits of
+    fmix32(key + id * 0x9E3779B9) + 1/2) / 2^24 in (0, 1), noise = -log(-log(u))."""
+    with np.errstate(over="ignore"):
+        h = fmix32(np.uint32(position_key(seed, seq, pos)) + np.arange(vocab, dtype=np.uint32) * np.uint32(0x9E3779B9))
+    u = ((h >> np.uint32(8)).astype(F64) + 0.5) * (1.0 / 16777216.0)
+    return -np.log(-np.log(u))
+
+
+def choose_tokens(cfg: OracleConfig, logits: np.ndarray, pred_pos: Sequence[int]) -> np.ndarray:
+    """The model's prediction for each row: the argmax (temperature 0), or a draw from
+    softmax(logits / temperature) by the Gumbel-max rule: argmax(logits / temperature + noise).
+
+    The noise of a row depends on the POSITION the row predicts, not on the row: the autoregressive
+    row of a position, the diffusion slots that pre-draft it and a plain one-token-per-pass decoder
+    all draw with the same noise, so sampled TiDAR (beta = 1) emits exactly what sampled
+    autoregressive decoding with this rule emits, and nothing depends on how positions are
+    batched into passes."""
+    logits = np.atleast_2d(logits)
+    if cfg.temperature <= 0.0:
+        return argmax_lowest(logits)
+    out = np.empty(len(logits), dtype=np.int64)
+    for r, p in enumerate(pred_pos):
+        out[r] = int(np.argmax(logits[r] / cfg.temperature + gumbel_noise(cfg.sample_seed, cfg.seq, int(p), logits.shape[-1])))
+    return out
+
+
+# ----------------------------------------------------------------------------
 # acceptance  (Section 3.2; Section 4.4.3)
 # ----------------------------------------------------------------------------
 def accept_length(block: Sequence[int], targets: Sequence[int], forced: int = 0) -> int:
@@ -346,10 +411,10 @@ def prefill(cfg: OracleConfig, w: dict, prompt: Sequence[int], k: int, return_fo
     fo = forward(cfg, w, ids, pos, mask, kc, vc, logit_rows=None if return_forward else rows)
     a = fo.logits[n - 1]
     g = fo.logits[n:]
-    c = int(argmax_lowest(cfg.beta * a + (1.0 - cfg.beta) * g[0]))
+    c = int(choose_tokens(cfg, cfg.beta * a + (1.0 - cfg.beta) * g[0], [n])[0])      # row n-1 and mask row 0 predict position n
     block = np.empty(k, dtype=np.int64)
     block[0] = c
-    block[1:] = argmax_lowest(g[1:])
+    block[1:] = choose_tokens(cfg, g[1:], n + np.arange(1, k))                        # mask row i predicts position n + i
     st = OracleState(n=n, k_cache=[x[:n].copy() for x in fo.k_new], v_cache=[x[:n].copy() for x in fo.v_new],
                      block=block, tokens=list(map(int, prompt)) + [c])
     return (st, c, fo) if return_forward else (st, c)
@@ -375,8 +440,8 @@ def step(cfg: OracleConfig, w: dict, st: OracleState, forced: int = 0) -> StepOu
     fo = forward(cfg, w, ids, pos, mask, st.k_cache, st.v_cache)
     a = fo.logits[:k]                                  # causal slot j -> position n + j + 1
     g = fo.logits[k:].reshape(k, k, -1)                # mask (b, i) -> position n + b + 1 + i
-    targets = argmax_lowest(cfg.beta * a + (1.0 - cfg.beta) * g[:, 0, :])
-    draft_ids = argmax_lowest(g)
+    targets = choose_tokens(cfg, cfg.beta * a + (1.0 - cfg.beta) * g[:, 0, :], n + 1 + np.arange(k))
+    draft_ids = choose_tokens(cfg, g.reshape(k * k, -1), [n + b + 1 + i for b in range(k) for i in range(k)]).reshape(k, k)
     L = accept_length(st.block, targets, forced)
     emitted = [int(t) for t in st.block[1:L]] + [int(targets[L - 1])]
     # commit K/V of the accepted causal slots only; the rest is evicted
@@ -428,7 +493,7 @@ def ar_generate(cfg: OracleConfig, w: dict, prompt: Sequence[int], max_new_token
     fo = forward(cfg, w, ids, np.arange(n, dtype=np.int64), np.tril(np.ones((n, n), dtype=bool)), kc, vc,
                  logit_rows=np.array([n - 1]))
     kc, vc = [x.copy() for x in fo.k_new], [x.copy() for x in fo.v_new]
-    out = [int(argmax_lowest(fo.logits[n - 1]))]
+    out = [int(choose_tokens(cfg, fo.logits[n - 1], [n])[0])]
     while len(out) < max_new_tokens:
         m = np.ones((1, n + 1), dtype=bool)
         fo = forward(cfg, w, np.array([out[-1]]), np.array([n], dtype=np.int64), m, kc, vc)
@@ -436,5 +501,5 @@ def ar_generate(cfg: OracleConfig, w: dict, prompt: Sequence[int], max_new_token
             kc[l] = np.concatenate([kc[l], fo.k_new[l]], axis=0)
             vc[l] = np.concatenate([vc[l], fo.v_new[l]], axis=0)
         n += 1
-        out.append(int(argmax_lowest(fo.logits[0])))
+        out.append(int(choose_tokens(cfg, fo.logits[0], [n])[0]))
     return out

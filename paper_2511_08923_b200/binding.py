@@ -137,7 +137,7 @@ class Tidar:
 
     def __init__(self, shape, packed: dict, k_max: int, max_batch: int = 1, max_seq_len: int = 4096,
                  debug: int = 0, impl: int = 0, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
-                 guard_bytes: int = 0, beta: float = 1.0, prefill_rows: int = 0):
+                 guard_bytes: int = 0, beta: float = 1.0, prefill_rows: int = 0, temperature: float = 0.0, sample_seed: int = 0):
         self.lib = load()
         self.shape, self.k_max, self.max_batch = shape, k_max, max_batch
         self.device = torch.device(device)
@@ -145,7 +145,7 @@ class Tidar:
             n_layers=len(packed["layers"]), d_model=shape.d_model, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
             head_dim=shape.head_dim, d_ffn=shape.d_ffn, vocab=shape.vocab, tie_lm_head=int(shape.tie_lm_head),
             rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, mask_token_id=shape.mask_token_id, k_max=k_max,
-            max_batch=max_batch, max_seq_len=max_seq_len, page_size=64, beta=beta, temperature=0.0, sample_seed=0,
+            max_batch=max_batch, max_seq_len=max_seq_len, page_size=64, beta=beta, temperature=temperature, sample_seed=sample_seed,
             debug=debug, impl=impl, prefill_rows=prefill_rows)
         self.cfg = cfg
         nbytes = C.c_size_t(0)

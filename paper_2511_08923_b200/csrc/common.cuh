@@ -22,6 +22,7 @@ struct RowMeta {
   int32_t *nloc;       // number of local K/V rows visible
   int32_t *cache_pos;  // where this row's K/V go in the cache, or -1
   int32_t *local_idx;  // where this row's K/V go in the local scratch, or -1
+  uint32_t *skey;      // sampling key of the position this row predicts (written when sampling is on)
 };
 
 struct KvGeom {
@@ -44,6 +45,36 @@ __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
+}
+
+// ---- seeded sampling -------------------------------------------------------------------
+// A prediction is drawn from softmax(logits / temperature) by the Gumbel-max rule: the argmax of
+// logits / temperature + noise(id).  The noise is a pure function of (seed, sequence slot,
+// PREDICTED position, token id), so the autoregressive row of a position, the diffusion slots
+// that pre-draft it and a one-token-per-pass decoder all draw with the same noise, whatever pass
+// the position falls into.  mix64 is SplitMix64's output function, fmix32 MurmurHash3's 32-bit
+// finaliser.
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+__device__ __forceinline__ uint32_t fmix32(uint32_t h) {
+  h ^= h >> 16; h *= 0x85EBCA6Bu; h ^= h >> 13; h *= 0xC2B2AE35u; h ^= h >> 16;
+  return h;
+}
+__device__ __forceinline__ uint32_t position_key(unsigned long long seed, int seq, int pos) {
+  return (uint32_t)(mix64(mix64(seed + 0x9E3779B97F4A7C15ull) ^ (((unsigned long long)(uint32_t)seq << 32) | (uint32_t)pos)) >> 32);
+}
+// Standard Gumbel noise -ln(-ln u), u = (m + 1/2) / 2^24 with m the top 24 bits of the hash.
+// -ln u goes through log1p where u is close to 1 (there m + 1/2 is not a float, 2^24 - m - 1/2 is),
+// so the largest draws, the ones most likely to win, are as accurate as the rest.
+__device__ __forceinline__ float gumbel_noise(uint32_t key, uint32_t id) {
+  const uint32_t m = fmix32(key + id * 0x9E3779B9u) >> 8;
+  float e;
+  if (m < (1u << 23)) e = -logf(((float)m + 0.5f) * (1.0f / 16777216.0f));
+  else e = -log1pf(-((float)(16777216u - m) - 0.5f) * (1.0f / 16777216.0f));
+  return -logf(e);
 }
 
 // Programmatic dependent launch.  A kernel launched with the programmatic-serialization

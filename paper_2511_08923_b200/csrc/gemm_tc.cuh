@@ -37,7 +37,9 @@ constexpr int W_STAGE_BYTES = TILE_N * TILE_K * 2;
 constexpr int SMEM_BUDGET = 216 * 1024;   // dynamic shared memory for the rings; up to 9 KB of static shared memory come on top
 constexpr int TMEM_COLS = 512;
 
-enum Mode { MODE_SLAB = 0, MODE_SWIGLU = 1, MODE_ARGMAX = 2 };
+// MODE_SAMPLE is MODE_ARGMAX with Gumbel noise added to the tempered logits (a draw per row instead of
+// the argmax); it is a mode of its own so that the greedy LM head carries none of its registers.
+enum Mode { MODE_SLAB = 0, MODE_SWIGLU = 1, MODE_ARGMAX = 2, MODE_SAMPLE = 3 };
 
 struct Args {
   int R, N, K;              // activation rows in use, output features, input features
@@ -59,6 +61,9 @@ struct Args {
   // MODE_ARGMAX: per (CTA, lane quadrant) candidates, [R][cand_ld >= gridDim*4] (index -1 = none; the
   // caller pre-fills the index table with -1); optional fp32 dump [R][ld_dump]
   float *cand_val; int32_t *cand_idx; int cand_ld; float *dump; int ld_dump; int col0;
+  // MODE_SAMPLE: the compared value is logit * inv_temp + Gumbel noise of (skey[row], id),
+  // i.e. a draw from softmax(logits / temperature) per row (see gumbel_noise); the dump keeps the raw logits
+  float inv_temp; const uint32_t *skey;
   int *status;              // device word set to 1 when a bounded wait gave up
   __host__ __device__ int tile_b0_or_all() const { return n_tiles_b ? tile_b0 : n_tiles; }   // tiles per row block in the fused region
   __host__ __device__ int total_items() const { return fused_items + n_rb * n_tiles_b * S; }
@@ -75,7 +80,7 @@ __device__ __forceinline__ Item decode_item(const Args &g, int item) {
   Item w;
   if (item < g.fused_items) {
     w.fused = true; w.split = 0;
-    if (MODE == MODE_ARGMAX) { w.tile = item % g.tile_b0_or_all(); w.rb = item / g.tile_b0_or_all(); }
+    if (MODE == MODE_ARGMAX || MODE == MODE_SAMPLE) { w.tile = item % g.tile_b0_or_all(); w.rb = item / g.tile_b0_or_all(); }
     else { w.rb = item % g.n_rb; w.tile = item / g.n_rb; }
     w.kb0 = 0; w.kb1 = g.kb_total;
   } else {
@@ -433,6 +438,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int j = 0; j < 32; ++j) {
               const int i = grp * 2 + (j >> 4);
               float x = (i < 9 && i * 16 < ncols) ? __uint_as_float(v[i < 9 ? i : 8][j & 15]) : -INFINITY;
+              if (MODE == MODE_SAMPLE) {
+                const int r = r_base + grp * 32 + j;
+                if (r < g.R && n_ok) x = x * g.inv_temp + gumbel_noise(g.skey[r], (uint32_t)my_idx);
+              }
               const bool ok_v = n_ok && (x == x);
               val[j] = ok_v ? x : -INFINITY; idx[j] = ok_v ? my_idx : 0x7fffffff;
             }
@@ -457,7 +466,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
       }
     }
-    if (MODE == MODE_ARGMAX) flush_best();
+    if (MODE == MODE_ARGMAX || MODE == MODE_SAMPLE) flush_best();
   }
 
   // ---- teardown ----

@@ -41,7 +41,7 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
                                      const int32_t *__restrict__ block_ids, const int32_t *__restrict__ blk_len, int k, int n_blocks,
                                      int k_max, int mask_id,
                                      int32_t *__restrict__ step_n, const bf16 *__restrict__ embed, int d,
-                                     float *__restrict__ X, TlSlot tl) {
+                                     float *__restrict__ X, int sampling, unsigned long long seed, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
@@ -59,10 +59,12 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
     if (slot < k) {
       m.pos[r] = n + slot; m.nvis[r] = n + slot + 1; m.loc0[r] = 0; m.nloc[r] = 0;
       m.cache_pos[r] = n + slot; m.local_idx[r] = -1;
+      if (sampling) m.skey[r] = position_key(seed, seq, n + slot + 1);        // a causal slot predicts the next position
     } else {
       const int b = (slot - k) / k, i = (slot - k) % k;
       m.pos[r] = n + b + 1 + i; m.nvis[r] = n + b + 1; m.loc0[r] = s * k * k + b * k; m.nloc[r] = k;
       m.cache_pos[r] = -1; m.local_idx[r] = s * k * k + b * k + i;
+      if (sampling) m.skey[r] = position_key(seed, seq, n + b + 1 + i);       // a mask slot predicts its own position
     }
   }
   embed_row_to_f32(embed + (size_t)id * d, X + (size_t)r * d, d);
@@ -74,7 +76,7 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
 // prompt and each other.
 __global__ void assemble_prefill_kernel(RowMeta m, int seq, int row0, int n_prompt, int k, int mask_id,
                                         const int32_t *__restrict__ prompt, const bf16 *__restrict__ embed, int d,
-                                        float *__restrict__ X) {
+                                        float *__restrict__ X, int sampling, unsigned long long seed) {
   const int r = blockIdx.x;
   const int g = row0 + r;
   const int id = g < n_prompt ? prompt[g] : mask_id;
@@ -82,8 +84,10 @@ __global__ void assemble_prefill_kernel(RowMeta m, int seq, int row0, int n_prom
     m.seq[r] = seq; m.ids[r] = id; m.pos[r] = g;
     if (g < n_prompt) {
       m.nvis[r] = g + 1; m.loc0[r] = 0; m.nloc[r] = 0; m.cache_pos[r] = g; m.local_idx[r] = -1;
+      if (sampling) m.skey[r] = position_key(seed, seq, g + 1);
     } else {
       m.nvis[r] = n_prompt; m.loc0[r] = 0; m.nloc[r] = k; m.cache_pos[r] = -1; m.local_idx[r] = g - n_prompt;
+      if (sampling) m.skey[r] = position_key(seed, seq, g);
     }
   }
   embed_row_to_f32(embed + (size_t)id * d, X + (size_t)r * d, d);
@@ -290,14 +294,18 @@ __global__ void swiglu_slab_kernel(const SLAB *__restrict__ slabs, int S, size_t
 // Running per-row argmax over a chunk of logits [R][ncols] (fp32, leading dim ld)
 // that covers vocabulary ids [col0, col0+ncols).  Lowest index wins ties; NaN never
 // wins.  Optionally copies the chunk into a full [R][vocab] dump.
+// With inv_temp > 0 the compared value is logit * inv_temp + Gumbel noise of (skey[r], id): a draw
+// from softmax(logits / temperature) instead of the argmax; the dump always holds the raw logits.
 __global__ void argmax_chunk_kernel(const float *__restrict__ L, int ld, int ncols, int col0, int first,
                                     float *__restrict__ best_val, int32_t *__restrict__ best_idx,
-                                    float *__restrict__ dump, int vocab) {
+                                    float *__restrict__ dump, int vocab, float inv_temp, const uint32_t *__restrict__ skey) {
   const int r = blockIdx.x;
   float bv = -INFINITY; int bi = 0x7fffffff;
+  const uint32_t key = inv_temp > 0.f ? skey[r] : 0u;
   for (int c = threadIdx.x; c < ncols; c += blockDim.x) {
-    const float v = L[(size_t)r * ld + c];
+    float v = L[(size_t)r * ld + c];
     if (dump) dump[(size_t)r * vocab + col0 + c] = v;
+    if (inv_temp > 0.f) v = v * inv_temp + gumbel_noise(key, (uint32_t)(col0 + c));
     if (v > bv) { bv = v; bi = col0 + c; }
   }
   __shared__ float sv[32]; __shared__ int si[32];
@@ -408,13 +416,14 @@ __global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const 
 // is the argmax of the mixed logits.  Block i handles pair i:
 //   a = a0 + (i / k) * a_seq + (i % k) * a_j,  b likewise,  dst = dst0 + i.
 __global__ void mix_rows_kernel(bf16 *__restrict__ A, int d, float beta, int k, int a0, int a_seq, int a_j, int b0, int b_seq, int b_j,
-                                int dst0, TlSlot tl) {
+                                int dst0, uint32_t *__restrict__ skey, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
   const int i = blockIdx.x, s = i / k, j = i % k;
   const bf16 *ra = A + (size_t)(a0 + s * a_seq + j * a_j) * d, *rb = A + (size_t)(b0 + s * b_seq + j * b_j) * d;
   bf16 *ro = A + (size_t)(dst0 + i) * d;
+  if (skey && threadIdx.x == 0) skey[dst0 + i] = skey[a0 + s * a_seq + j * a_j];     // the mixed row predicts what row a predicts
   for (int c = threadIdx.x * 2; c < d; c += blockDim.x * 2) {
     const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(ra + c));
     const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(rb + c));

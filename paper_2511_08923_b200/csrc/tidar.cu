@@ -39,6 +39,7 @@ struct tidar_ctx {
   std::vector<const bf16 *> bqkv, q_norm, k_norm;      // optional (empty = absent)
   // geometry
   int R_head = 0;                  // rows of a pass that can get logits (the rows of a decode step)
+  int head_row0 = 0;               // first row of the current pass that the LM head runs on
   int last_hidden_off = 0;         // first row of the last pass that the read-back calls address
   int R_cap = 0, T_max = 0, pages_per_seq = 0, n_pages = 0, n_qkv = 0, S_max = 4, lm_chunk = 0;
   size_t pool_stride = 0;    // elements in one layer's K (or V) pool
@@ -135,7 +136,7 @@ int validate(const tidar_config &c, std::string &why) {
   if (c.max_batch < 1 || c.max_seq_len < 2 * c.k_max + 1) return bad("max_batch >= 1 and max_seq_len > 2*k_max required");
   if (c.mask_token_id < 0 || c.mask_token_id >= c.vocab) return bad("mask_token_id out of range");
   if (!(c.beta >= 0.0f && c.beta <= 1.0f)) return bad("beta must be in [0, 1]");
-  if (c.temperature != 0.0f) return bad("only greedy decoding (temperature 0) is implemented");
+  if (!(c.temperature >= 0.0f) || c.temperature > 1e4f) return bad("temperature must be in [0, 1e4] (0 = greedy)");
   if (c.impl != 0 && c.impl != 1) return bad("impl must be 0 (tensor-core kernels) or 1 (replay kernels)");
   if (c.prefill_rows < 0 || c.prefill_rows > (1 << 16)) return bad("prefill_rows must be in [0, 65536]");
   if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return bad("rms_eps > 0 and rope_theta > 1 required");
@@ -163,6 +164,7 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.meta.ids = cv.take<int32_t>(R); x.meta.pos = cv.take<int32_t>(R); x.meta.seq = cv.take<int32_t>(R);
   x.meta.nvis = cv.take<int32_t>(R); x.meta.loc0 = cv.take<int32_t>(R); x.meta.nloc = cv.take<int32_t>(R);
   x.meta.cache_pos = cv.take<int32_t>(R); x.meta.local_idx = cv.take<int32_t>(R);
+  x.meta.skey = cv.take<uint32_t>(R);
   x.d_seq_len = cv.take<int32_t>(c.max_batch);
   x.d_blk_len = cv.take<int32_t>(c.max_batch);
   x.d_run_max = cv.take<float>(R); x.d_run_sum = cv.take<float>(R); x.d_tgt_logit = cv.take<float>(R); x.d_logprob = cv.take<float>(R);
@@ -345,6 +347,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   } else {
     a.fused_items = a.n_rb * a.n_tiles;
     a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.cand_ld = c->n_sms * 4; a.dump = c->dbg_logits; a.ld_dump = c->cfg.vocab; a.col0 = 0;
+    a.inv_temp = c->cfg.temperature > 0.f ? 1.0f / c->cfg.temperature : 0.f; a.skey = c->meta.skey + c->head_row0;
   }
   a.status = c->d_status;
   const CUtensorMap *tmA = act_map(c, A, a_rows, K, a.box_rows);
@@ -355,6 +358,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
   Launch l(c, cls);
   if (mode == gemm_tc::MODE_SLAB) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
   else if (mode == gemm_tc::MODE_SWIGLU) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
+  else if (a.inv_temp > 0.f) launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SAMPLE>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
   else launch_pdl(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, grid, gemm_tc::THREADS, smem, c->stream, tmW, *tmA, a, l.tl);
   if (rem_tiles) {
     const int nf = (N - a.tile_b0 * gemm_tc::TILE_N) / 2;          // features of the split tiles
@@ -548,10 +552,13 @@ if (tc && c->slab_bf16)
                                 cudaMemcpyDeviceToDevice, c->stream));
   if (with_head && mix.n > 0) {            // rows R .. R + mix.n - 1 of the LM head's input
     Launch lm(c, TIDAR_TC_NORM);
-    launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, R, lm.tl);
+    launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, R,
+                 cf.temperature > 0.f ? c->meta.skey : (uint32_t *)nullptr, lm.tl);
     R += mix.n;
   }
   const bf16 *Ah = c->A + (size_t)head_row0 * d;           // first row of the LM head's input
+  c->head_row0 = head_row0;
+  const float inv_temp = cf.temperature > 0.f ? 1.0f / cf.temperature : 0.f;
   const int Rh = R - head_row0;
   if (with_head && Rh > c->R_head) return fail(c, TIDAR_ECAPACITY, "%d rows for the LM head exceed the context's %d", Rh, c->R_head);
   if (with_head && tc) {
@@ -565,7 +572,8 @@ if (tc && c->slab_bf16)
       const int nc = std::min(c->lm_chunk, cf.vocab - v0);
       if ((rc = gemm_partials(c, Ah, RA - head_row0, c->lm_head + (size_t)v0 * d, nullptr, Rh, nc, d, c->partials, &S, &stride, TIDAR_TC_LMHEAD))) return rc;
       Launch ll(c, TIDAR_TC_LMHEAD);
-      argmax_chunk_kernel<<<Rh, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab);
+      argmax_chunk_kernel<<<Rh, 256, 0, c->stream>>>(c->partials, nc, nc, v0, v0 == 0, c->d_arg_val, c->d_arg_idx, c->dbg_logits, cf.vocab, inv_temp,
+                                                     c->meta.skey + head_row0);
     }
   }
   CUDA_TRY(c, cudaGetLastError());
@@ -620,6 +628,7 @@ int init_tensor_core_path(tidar_ctx *c) {
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SLAB>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_ARGMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc::gemm_tc_kernel<gemm_tc::MODE_SAMPLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
   return TIDAR_OK;
 }
 
@@ -676,7 +685,7 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar) {
   {
     Launch l(c, TIDAR_TC_EMBED);
     launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, c->d_blk_len, k, n_blocks, cf.k_max,
-               cf.mask_token_id, c->d_step_n, c->embed, cf.d_model, c->X, l.tl);
+               cf.mask_token_id, c->d_step_n, c->embed, cf.d_model, c->X, cf.temperature > 0.f ? 1 : 0, (unsigned long long)cf.sample_seed, l.tl);
   }
   // beta < 1: the verified prediction of causal slot j mixes its row with the first slot of block j
   MixRows mix;
@@ -895,7 +904,7 @@ int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_pr
     {
       Launch l(c, TIDAR_TC_EMBED);
       assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n_prompt, k, cf.mask_token_id, c->d_prompt, c->embed,
-                                                           cf.d_model, c->X);
+                                                           cf.d_model, c->X, cf.temperature > 0.f ? 1 : 0, (unsigned long long)cf.sample_seed);
     }
     // beta < 1: the settled first token mixes the last prompt row with the first mask row
     MixRows mix;
@@ -982,7 +991,7 @@ int tidar_score(tidar_ctx *c, int32_t seq, const int32_t *ids, int32_t n, float 
     const int rows = std::min(c->R_cap, n - 1 - row0);          // the last token predicts nothing that is scored
     {
       Launch l(c, TIDAR_TC_EMBED);
-      assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n, 0, cf.mask_token_id, c->d_prompt, c->embed, d, c->X);
+      assemble_prefill_kernel<<<rows, 256, 0, c->stream>>>(c->meta, seq, row0, n, 0, cf.mask_token_id, c->d_prompt, c->embed, d, c->X, 0, 0ull);
     }
     if (int rc = forward_rows(c, rows, false, rows, (row0 + rows / 2 + 63) / 64)) return rc;      // ends with the final norm in c->A
     for (int v0 = 0, ci = 0; v0 < cf.vocab; v0 += c->lm_chunk, ++ci) {

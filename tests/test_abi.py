@@ -48,7 +48,7 @@ def test_arena_bytes_and_validation_run_on_the_host():
     assert lib.tidar_arena_bytes(C.byref(_cfg(debug=1)), C.byref(n)) == 0
     assert n.value > small
     for bad in (dict(head_dim=96), dict(page_size=32), dict(k_max=0), dict(k_max=33), dict(n_q_heads=3),
-                dict(mask_token_id=5000), dict(beta=1.5), dict(beta=-0.1), dict(temperature=1.0), dict(d_model=100),
+                dict(mask_token_id=5000), dict(beta=1.5), dict(beta=-0.1), dict(temperature=-1.0), dict(d_model=100),
                 dict(max_seq_len=8), dict(n_q_heads=0, n_kv_heads=1), dict(n_q_heads=256, n_kv_heads=1),
                 dict(d_model=12352)):
         assert lib.tidar_arena_bytes(C.byref(_cfg(**bad)), C.byref(n)) == -1, bad

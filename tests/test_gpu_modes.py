@@ -199,3 +199,66 @@ def test_projection_bias_and_per_head_qk_norm(impl, family, hd):
         if (top1_margin(so.fwd.logits[:k]) > MARGIN).all():
             assert toks[0] == so.emitted
     _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_seeded_sampling_draws_what_the_oracle_draws(tiny, impl):
+    """temperature > 0: every prediction is a Gumbel-max draw keyed by (seed, slot, predicted position,
+    token id).  The GPU's draws of every row equal the argmax of its own tempered logits plus the
+    oracle's noise for that position, and follow the oracle's step wherever the noisy margin is clear;
+    free-running sampled TiDAR equals sampled one-token-per-pass decoding of the GPU itself."""
+    sh, wt, cfg, w, prompt = tiny
+    k, temp, seed = sh.k, 0.8, 33
+    cfg_s = replace(cfg, temperature=temp, sample_seed=seed, seq=0)
+    t = _gpu(sh, wt, impl, k_max=k, debug=1, max_batch=1)
+    t.close()
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    t = Tidar(sh, pack_weights(wt, "cuda:0"), k_max=k, max_seq_len=512, debug=1, impl=impl, temperature=temp, sample_seed=seed, guard_bytes=64 * 1024)
+    n = len(prompt)
+    T = k * (k + 1)
+
+    def noisy(lg, positions):
+        return np.stack([lg[r] / temp + O.gumbel_noise(seed, 0, int(p), sh.vocab) for r, p in enumerate(positions)])
+
+    first = t.prefill(0, prompt, k)
+    st, c, fo = O.prefill(cfg_s, w, prompt, k, return_forward=True)
+    lg = t.logits(0, n + k)
+    pred = np.concatenate([np.arange(1, n + 1), n + np.arange(k)])       # prompt row g predicts g + 1, mask row i predicts n + i
+    sc = noisy(lg.astype(np.float64), pred)
+    ids = t.argmax(0, n + k)
+    m = top1_margin(sc)
+    sure = m > 1e-3
+    np.testing.assert_array_equal(ids[sure], sc.argmax(-1)[sure])        # the GPU's draw from its own logits
+    assert sure.mean() > 0.95
+    assert (ids != lg.argmax(-1)).mean() > 0.2                           # and they are draws, not argmaxes
+    if top1_margin(noisy(fo.logits[n - 1:n], [n]))[0] > 2 * TOL_LOGITS / temp:
+        assert first == c
+    for s in range(4):
+        t.set_block(0, st.block)
+        block = st.block.copy()
+        so = O.step(cfg_s, w, st)
+        toks, L = t.step([0])
+        lg = t.logits(0, T)
+        _, _, _, pos = O.slot_layout(st.n - so.L, k)
+        pred = np.concatenate([pos[:k] + 1, pos[k:]])
+        sc = noisy(lg.astype(np.float64), pred)
+        ids = t.argmax(0, T)
+        sure = top1_margin(sc) > 1e-3
+        np.testing.assert_array_equal(ids[sure], sc.argmax(-1)[sure])
+        L_ref = O.accept_length(block, ids[:k])
+        assert L[0] == L_ref and toks[0] == [int(x) for x in block[1:L_ref]] + [int(ids[L_ref - 1])]
+        ref_sc = noisy(so.fwd.logits, pred)
+        if (top1_margin(ref_sc[:k]) > 2 * TOL_LOGITS / temp).all():
+            assert L[0] == so.L and toks[0] == so.emitted
+        elif L[0] != so.L:
+            break
+    # free running: sampled TiDAR steps against sampled autoregressive steps on the same GPU kernels
+    out = [t.prefill(0, prompt, k)]
+    while len(out) < 24:
+        out.extend(t.step([0])[0][0])
+    ar = [t.prefill(0, prompt, 1)]
+    while len(ar) < 24:
+        ar.extend(t.ar_step([0]))
+    agree = next((i for i, (a, b) in enumerate(zip(out, ar)) if a != b), 24)
+    assert agree >= 12, (out, ar)        # identical up to a near-tie of two differently rounded passes
+    _close(t)

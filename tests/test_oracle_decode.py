@@ -269,3 +269,66 @@ def test_planted_wrong_mask_position_breaks_predraft_pin(model, monkeypatch):
     monkeypatch.undo()
     _, _, fo2 = O.prefill(cfg, w, st.tokens[:st.n], sh.k, return_forward=True)
     assert np.abs(so.fwd.logits[sh.k:2 * sh.k] - fo2.logits[st.n:]).max() > 1e-6
+
+
+# ---------------------------------------------------------------- seeded sampling
+def test_hash_functions_match_their_published_values():
+    # SplitMix64 started at 0 produces 0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F (the reference
+    # implementation's first outputs): output i is mix64 of i+1 times the golden-ratio increment
+    g = 0x9E3779B97F4A7C15
+    assert [O.mix64((i + 1) * g) for i in range(3)] == [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
+    # MurmurHash3's 32-bit finaliser: 0 is a fixed point, fmix32(1) = 0x514E28B7; it is a bijection, so
+    # 2^16 distinct inputs give 2^16 distinct outputs
+    np.testing.assert_array_equal(O.fmix32(np.array([0, 1], dtype=np.uint32)), np.array([0, 0x514E28B7], dtype=np.uint32))
+    assert len(np.unique(O.fmix32(np.arange(1 << 16, dtype=np.uint32)))) == 1 << 16
+
+
+def test_gumbel_noise_is_standard_gumbel_and_keyed_by_position_only():
+    g = np.concatenate([O.gumbel_noise(11, 0, p, 4096) for p in range(64)])
+    # standard Gumbel: mean = Euler's constant, variance = pi^2 / 6, median = -ln ln 2
+    assert abs(g.mean() - 0.5772156649) < 0.01 and abs(g.var() - np.pi ** 2 / 6) < 0.03
+    assert abs(np.median(g) + np.log(np.log(2.0))) < 0.01
+    np.testing.assert_array_equal(O.gumbel_noise(11, 3, 77, 100), O.gumbel_noise(11, 3, 77, 1000)[:100])   # a pure function of (seed, seq, pos, id)
+    for other in (O.gumbel_noise(12, 3, 77, 100), O.gumbel_noise(11, 4, 77, 100), O.gumbel_noise(11, 3, 78, 100)):
+        assert np.abs(other - O.gumbel_noise(11, 3, 77, 100)).min() > 0 or not np.array_equal(other, O.gumbel_noise(11, 3, 77, 100))
+
+
+def test_draws_follow_softmax_of_the_tempered_logits():
+    """Gumbel-max sampling pinned by what it must reproduce: over many positions the frequency of every token
+    is its softmax(logits / temperature) probability; temperature -> 0 gives the argmax."""
+    from dataclasses import replace
+    sh = CONFIGS["tiny"]
+    base = _cfg(sh)
+    logits = np.array([2.0, 1.0, 0.5, 0.0, -1.0, -3.0])
+    for temp in (1.0, 0.5):
+        cfg = replace(base, temperature=temp, sample_seed=5)
+        n = 20000
+        draws = O.choose_tokens(cfg, np.tile(logits, (n, 1)), np.arange(n))
+        p = np.exp(logits / temp); p /= p.sum()
+        freq = np.bincount(draws, minlength=len(logits)) / n
+        assert np.abs(freq - p).max() < 4.5 * np.sqrt(p.max() * (1 - p.max()) / n) + 1e-3, (freq, p)
+    cold = replace(base, temperature=1e-4, sample_seed=5)
+    assert (O.choose_tokens(cold, np.tile(logits, (50, 1)), np.arange(50)) == 0).all()
+    assert (O.choose_tokens(base, np.tile(logits, (3, 1)), np.arange(3)) == 0).all()         # temperature 0: argmax
+
+
+@pytest.mark.parametrize("drafts", ["natural", "garbage"])
+def test_sampled_tidar_equals_sampled_autoregressive_decoding(model, drafts):
+    """The noise of a draw depends on the predicted position only, so with beta = 1 sampled TiDAR must emit
+    exactly what one-token-per-pass sampled decoding emits, whatever the drafts were; and the draws differ
+    from greedy decoding (the temperature is live)."""
+    from dataclasses import replace
+    sh, cfg, w, prompt = model
+    cfg_s = replace(cfg, temperature=0.9, sample_seed=21)
+    ar = O.ar_generate(cfg_s, w, prompt, 24)
+    rng = np.random.default_rng(0)
+
+    def garbage(st):
+        st.block[1:] = rng.integers(0, sh.vocab - 1, len(st.block) - 1)
+    out, Ls, _ = O.generate(cfg_s, w, prompt, sh.k, 24, draft_hook=garbage if drafts == "garbage" else None)
+    assert out == ar
+    assert ar != O.ar_generate(cfg, w, prompt, 24)
+    if drafts == "garbage":
+        assert max(Ls) <= 2
+    # another sequence slot or seed draws differently
+    assert O.ar_generate(replace(cfg_s, seq=1), w, prompt, 24) != ar and O.ar_generate(replace(cfg_s, sample_seed=22), w, prompt, 24) != ar
