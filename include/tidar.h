@@ -253,6 +253,11 @@ int tidar_debug_count_attention_tiles(tidar_ctx *ctx, int32_t on, uint64_t *visi
 int tidar_debug_set_timeline(tidar_ctx *ctx, int32_t on);
 int tidar_debug_get_timeline(tidar_ctx *ctx, float *class_ms /*host,[TIDAR_TC_COUNT]*/, float *busy_ms /*host, or NULL*/,
                              float *span_ms /*host, or NULL*/);
+/* Exercises the bounded wait the tensor-core kernels are built on: enqueues a one-thread kernel
+ * that waits, for at most limit_polls polls (a few milliseconds at 2^14), on a barrier that
+ * nothing arrives on, gives up and sets the status word.  tidar_sync then returns
+ * TIDAR_EDEVICE_TIMEOUT and the context stays usable.  impl 0 only.                       */
+int tidar_debug_wait_probe(tidar_ctx *ctx, int32_t limit_polls);
 /* Test hook for the error plumbing: writes `value` into the device status word that the
  * kernels set when a bounded wait gives up.  The next tidar_step / tidar_prefill /
  * tidar_sync then reports TIDAR_EDEVICE_TIMEOUT exactly as after a real timeout.  No
@@ -287,7 +292,8 @@ int tidar_attention(tidar_ctx *ctx, const void *q, const void *k_pages, const vo
 /* ---- one projection alone (microbenchmark and unit parity) ----------------------------
  * out[r][n] = sum_k A[r][k] * W[n][k]: the weight-streaming small-M GEMM every projection
  * of a step uses (QKV, O, gate/up, down, LM head; the step's k(k+1) token slots share one
- * pass over the weights: paper Section 1, "free token slots").
+ * pass over the weights: paper Section 1, where extra token slots cost next to nothing while
+ * the pass is bound by loading the weights).
  *   A [R][K] bf16, W [N][K] bf16, out [R][N] fp32, all DEVICE, row-major, 16-byte aligned;
  *   K a multiple of 64.  splits: K splits (1..8), 0 = the library's own choice; partial
  *   sums are combined in a fixed order, so the result is deterministic.

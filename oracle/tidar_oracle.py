@@ -7,7 +7,7 @@ shares no code with it and never calls it.
 
 What the paper fixes and where (all citations are to the paper):
 
-* Section 1, "at each generation step ... three sections": a step's forward
+* Section 1 (what one generation step feeds the model): a step's forward
   carries the cached prefix, the tokens proposed by the previous step, and the
   mask-token slots that pre-draft the next step.
 * Section 3.3 footnote: a step has ``q_len = k * (1 + k)`` token slots for a
@@ -73,8 +73,8 @@ class OracleConfig:
     beta: float = 1.0
     # "f64": nothing is rounded (the definition).  "bf16": the activations a bf16 decoder keeps between
     # its operators (normed inputs of the projections, Q, K, V after RoPE, the attention output, the
-    # SwiGLU output) are rounded to bfloat16 where they are stored; the paper trains and runs in
-    # "standard BFloat 16" (Section 4.1).  All arithmetic stays float64 in both modes.
+    # SwiGLU output) are rounded to bfloat16 where they are stored; the paper trains and runs the
+    # model in bfloat16 (Section 4.1).  All arithmetic stays float64 in both modes.
     act_dtype: str = "f64"
     # temperature 0: every prediction is the argmax (the hot path).  temperature > 0: every prediction is
     # a draw from softmax(logits / temperature), taken with noise that depends only on (sample_seed,

@@ -87,6 +87,7 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_sync": (C.c_int, [ctxp]),
         "tidar_attention_static": (C.c_int, [VP, VP, VP, I32, VP, I32, VP, VP, VP, VP, I32, I32, I32, I32, I32, VP]),
         "tidar_debug_force_status": (C.c_int, [ctxp, I32]),
+        "tidar_debug_wait_probe": (C.c_int, [ctxp, I32]),
         "tidar_debug_count_attention_tiles": (C.c_int, [ctxp, I32, P(C.c_uint64)]),
         "tidar_debug_set_timeline": (C.c_int, [ctxp, I32]),
         "tidar_debug_get_timeline": (C.c_int, [ctxp, P(C.c_float), P(C.c_float), P(C.c_float)]),
@@ -304,6 +305,10 @@ class Tidar:
         P16 = C.POINTER(C.c_uint16)
         self._check(self.lib.tidar_debug_get_kv(self.ctx, seq, layer, pos0, npos, k.ctypes.data_as(P16), v.ctypes.data_as(P16)))
         return k, v
+
+    def wait_probe(self, limit_polls: int = 1 << 14):
+        """Enqueue a kernel whose bounded wait runs out (see tidar_debug_wait_probe)."""
+        self._check(self.lib.tidar_debug_wait_probe(self.ctx, int(limit_polls)))
 
     def force_status(self, value: int):
         """Test hook: pretend a kernel's bounded wait gave up (see tidar_debug_force_status)."""

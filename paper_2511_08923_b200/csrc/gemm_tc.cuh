@@ -5,8 +5,8 @@
 //
 // A decode step has only k*(k+1) token slots per sequence (paper Section 3.3 footnote),
 // so every projection is a GEMM with a small row count and a weight matrix that is read
-// exactly once: the "free token slots" regime of the paper (Section 1; figure "Latency
-// Scaling").  The kernel therefore puts the WEIGHT rows on the 128 TMEM lanes (the MMA M
+// exactly once: the regime in which, by the paper's argument, extra token slots are nearly free
+// (Section 1; figure "Latency Scaling").  The kernel therefore puts the WEIGHT rows on the 128 TMEM lanes (the MMA M
 // dimension) and the activation rows on the MMA N dimension (up to 288 = two instructions
 // of up to 144 columns), so no tensor-core work is wasted on padding rows.
 //

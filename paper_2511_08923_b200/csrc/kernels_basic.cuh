@@ -2,6 +2,7 @@
 // draft/verify and KV commit kernels of the TiDAR decode step.
 #pragma once
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 // Four consecutive split-K partial sums starting at p (fp32 or bf16 slabs).
 template <typename T> __device__ __forceinline__ float4 load4(const T *p);
@@ -529,5 +530,25 @@ __global__ void kv_gather_kernel(const bf16 *__restrict__ Kp, const bf16 *__rest
   for (int c = threadIdx.x; c < g.head_dim; c += blockDim.x) {
     ko[((size_t)p * g.n_kv_heads + kvh) * g.head_dim + c] = Kp[off + c];
     vo[((size_t)p * g.n_kv_heads + kvh) * g.head_dim + c] = Vp[off + c];
+  }
+}
+
+// Probe of the bounded wait every tensor-core kernel is built on: one thread waits, with a
+// short limit, on an mbarrier that nothing will ever arrive on, gives up, and reports it through
+// the status word, exactly as a kernel whose producer went missing would.  Nothing hangs: the
+// wait is the same bounded loop, only shorter.  waited[0] receives the polls it took.
+__global__ void wait_probe_kernel(uint32_t limit, int *status, int *waited) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    sm100::mbar_init(sm100::smem_u32(&bar), 1);
+    sm100::fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool ok = sm100::mbar_wait(sm100::smem_u32(&bar), 0u, &abort_flag, limit);      // phase 0 never completes
+    waited[0] = ok ? 0 : (int)limit;
+    if (!ok && abort_flag) atomicExch(status, 9);
   }
 }

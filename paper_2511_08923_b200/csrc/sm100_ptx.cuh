@@ -36,10 +36,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when it gave up, or when another thread of the CTA
-// already gave up (*abort_flag != 0; the flag lives in shared memory).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+// Bounded wait.  Returns false when it gave up (after `limit` failed polls), or when another
+// thread of the CTA already gave up (*abort_flag != 0; the flag lives in shared memory).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t limit = WAIT_LIMIT) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i >= 128) {
       __nanosleep(i < 4096 ? 20 : 200);

@@ -1114,6 +1114,15 @@ int tidar_debug_get_kv(tidar_ctx *c, int32_t seq, int32_t layer, int32_t pos0, i
   return TIDAR_OK;
 }
 
+int tidar_debug_wait_probe(tidar_ctx *c, int32_t limit_polls) {
+  if (!c) return TIDAR_EINVAL;
+  if (c->cfg.impl != 0) return fail(c, TIDAR_EINVAL, "the bounded waits exist in the tensor-core kernels only");
+  if (limit_polls < 1 || limit_polls > (1 << 20)) return fail(c, TIDAR_EINVAL, "limit_polls must be in [1, 2^20]");
+  wait_probe_kernel<<<1, 32, 0, c->stream>>>((uint32_t)limit_polls, c->d_status, c->d_status + 8);
+  CUDA_TRY(c, cudaGetLastError());
+  return TIDAR_OK;
+}
+
 int tidar_debug_force_status(tidar_ctx *c, int32_t value) {
   if (!c) return TIDAR_EINVAL;
   CUDA_TRY(c, cudaMemcpyAsync(c->d_status, &value, sizeof(int), cudaMemcpyHostToDevice, c->stream));

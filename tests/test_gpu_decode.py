@@ -380,6 +380,13 @@ def test_device_timeout_status_is_reported_and_sequences_released(tiny, impl):
         t.sync()
     assert e.value.code == -5
     t.sync()                                        # the word was cleared by the report
+    # a real bounded wait that runs out: a barrier nothing arrives on, a limit of 2^14 polls
+    t.wait_probe(1 << 14)
+    with pytest.raises(TidarError) as e:
+        t.sync()
+    assert e.value.code == -5 and "status 9" in str(e.value)
+    t.prefill(0, prompt, k)                         # the context is still usable
+    assert t.step([0], forced=[1])[1] == [1]
     _close(t)
 
 
