@@ -320,8 +320,9 @@ int tidar_sync(tidar_ctx *ctx);
  * The call performs no cudaMalloc/cudaFree and calls no allocating routine.
  *   - It always runs the plain CUDA-core kernel (one warp per row and query head, fp32
  *     accumulation, K/V re-read once per query head, no tile skipping), not the
- *     tensor-core kernel: correct and allocation-free, not fast (about 30 times slower
- *     than tidar_attention with impl 0 at a thousand cached positions).
+ *     tensor-core kernel: correct and allocation-free, not fast (measured at 32 / 8 heads,
+ *     k = 16: 1.1 ms against 28 us for tidar_attention with impl 0 at a thousand cached
+ *     positions, 4.2 ms against 45 us at four thousand).
  *   - Limit: n_seqs * k * (k+1) <= 4352 rows (16 sequences at k = 16); beyond that the
  *     call returns TIDAR_ECAPACITY and launches nothing.  page_size is 64.
  *   - Each GPU that loads the library holds the table (85 KiB) until the process exits.
