@@ -172,6 +172,18 @@ int tidar_step_k(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t 
                  const int32_t *forced_accept /*host or NULL*/, int32_t *out_tokens /*host,[n_seqs][k_max]*/,
                  int32_t *out_n /*host,[n_seqs]*/);
 
+/* A decode step in which listed sequence i uses its own block length ks[i] (host, [n_seqs], each in
+ * [1, k_max]); the paper's Section 5 lets the block length follow the compute profile and nothing in
+ * the method ties the sequences of a batch to one length.  The pass has sum_i ks[i]*(ks[i]+1) token
+ * slots, sequence after sequence.  Per sequence the results are those of tidar_step_k with that
+ * sequence's length (same tokens; hidden states up to the rounding of a different row count).
+ * forced_accept[i] in [0, ks[i]].  Equal lengths take tidar_step_k's path; different lengths are
+ * launched kernel by kernel (no captured graph) and need beta == 1 (TIDAR_EINVAL otherwise).
+ * out_tokens / out_n as in tidar_step.                                                        */
+int tidar_step_ks(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs, const int32_t *ks /*host,[n_seqs]*/,
+                  const int32_t *forced_accept /*host or NULL*/, int32_t *out_tokens /*host,[n_seqs][k_max]*/,
+                  int32_t *out_n /*host,[n_seqs]*/);
+
 /* The block length that keeps a step of n_seqs sequences within row_budget token slots:
  * the largest k <= k_max with n_seqs*k*(k+1) <= row_budget (at least 1).  row_budget <= 0
  * selects 288, one row block of the projection kernels, about where the 8B-class step

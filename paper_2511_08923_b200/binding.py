@@ -66,6 +66,7 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_step_async": (C.c_int, [ctxp, P(I32), I32, P(I32)]),
         "tidar_step_wait": (C.c_int, [ctxp, P(I32), P(I32)]),
         "tidar_step_k": (C.c_int, [ctxp, P(I32), I32, I32, P(I32), P(I32), P(I32)]),
+        "tidar_step_ks": (C.c_int, [ctxp, P(I32), I32, P(I32), P(I32), P(I32), P(I32)]),
         "tidar_ar_step": (C.c_int, [ctxp, P(I32), I32, P(I32)]),
         "tidar_ridge_k": (C.c_int, [ctxp, I32, I32]),
         "tidar_score": (C.c_int, [ctxp, I32, P(I32), I32, P(C.c_float)]),
@@ -229,6 +230,18 @@ class Tidar:
         toks = np.empty((len(s), self.k_max), dtype=np.int32)
         n = np.empty(len(s), dtype=np.int32)
         self._check(self.lib.tidar_step_k(self.ctx, _ip(s), len(s), k, _ip(f) if f is not None else None, _ip(toks), _ip(n)))
+        return [toks[i, :n[i]].tolist() for i in range(len(s))], n.tolist()
+
+    def step_ks(self, seqs: Sequence[int], ks: Sequence[int], forced: Optional[Sequence[int]] = None):
+        """A decode step in which each listed sequence uses its own block length (see tidar_step_ks)."""
+        s = _i32(seqs)
+        kk = _i32(ks)
+        if len(kk) != len(s):
+            raise ValueError("one block length per listed sequence")
+        f = _i32(forced) if forced is not None else None
+        toks = np.empty((len(s), self.k_max), dtype=np.int32)
+        n = np.empty(len(s), dtype=np.int32)
+        self._check(self.lib.tidar_step_ks(self.ctx, _ip(s), len(s), _ip(kk), _ip(f) if f is not None else None, _ip(toks), _ip(n)))
         return [toks[i, :n[i]].tolist() for i in range(len(s))], n.tolist()
 
     def ar_step(self, seqs: Sequence[int]) -> List[int]:

@@ -37,6 +37,10 @@ struct Args {
   int rows_per_group;       // slots per sequence group (k(k+1) for a step; R for a first pass)
   int tiles_per_group;      // ceil(rows_per_group / spt)
   int n_groups;
+  // Groups of different sizes (a step whose sequences use different block lengths): query tile t
+  // covers rows [tile_row0[t], tile_row0[t] + spt) of the group that ends at tile_rend[t]; null =
+  // equal groups, derived from rows_per_group.  n_tiles = number of query tiles in either case.
+  const int32_t *tile_row0, *tile_rend; int n_tiles;
   int spt;                  // slots per query tile = 128 / G
   int G, Hq, Hkv;
   int splits;
@@ -95,9 +99,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   int w = blockIdx.x;
   const int sp = w % a.splits; w /= a.splits;
   const int kvh = w % a.Hkv; w /= a.Hkv;
-  const int tile = w % a.tiles_per_group; const int grp = w / a.tiles_per_group;
-  const int row0 = grp * a.rows_per_group + tile * a.spt;              // first slot of the tile
-  const int row_end = min((grp + 1) * a.rows_per_group, a.R);          // slots of this group end here
+  int row0, row_end;                                                   // first slot of the tile; slots of its group end at row_end
+  if (a.tile_row0) { row0 = a.tile_row0[w]; row_end = a.tile_rend[w]; }
+  else {
+    const int tile = w % a.tiles_per_group, grp = w / a.tiles_per_group;
+    row0 = grp * a.rows_per_group + tile * a.spt;
+    row_end = min((grp + 1) * a.rows_per_group, a.R);
+  }
   const int rows_used = a.spt * a.G;                                   // MMA rows that carry data
 
   if (threadIdx.x == 0) {

@@ -36,19 +36,30 @@ __device__ __forceinline__ void embed_row_to_f32(const bf16 *__restrict__ e, flo
 // The step may use a block length k that differs from the one the previous pass left
 // (blk_len[seq] valid entries): drafts the sequence does not have are fed as [MASK]
 // and can never be accepted (see verify_select_kernel).
+// The listed sequences may use different block lengths in one step: step_k[s] is sequence s's,
+// step_off[s] its first row and step_loc[s] its first step-local K/V row (null: all use k).
 // One block per row; also snapshots n into step_n for the commit kernel.
 // ---------------------------------------------------------------------------
+struct StepLayout { const int32_t *k, *off, *loc; int n_seqs; };     // per listed sequence; k == null: uniform
+
 __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ seq_len,
                                      const int32_t *__restrict__ block_ids, const int32_t *__restrict__ blk_len, int k, int n_blocks,
-                                     int k_max, int mask_id,
+                                     StepLayout lay, int k_max, int mask_id,
                                      int32_t *__restrict__ step_n, const bf16 *__restrict__ embed, int d,
                                      float *__restrict__ X, int sampling, unsigned long long seed, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
-  const int T = k * (n_blocks + 1);
   const int r = blockIdx.x;
-  const int s = r / T, slot = r % T;
+  int s, slot, loc_base;
+  if (lay.k) {                                   // per-sequence block lengths: find the sequence this row belongs to
+    s = 0;
+    while (s + 1 < lay.n_seqs && r >= lay.off[s + 1]) ++s;
+    k = lay.k[s]; n_blocks = k; slot = r - lay.off[s]; loc_base = lay.loc[s];
+  } else {
+    const int T = k * (n_blocks + 1);
+    s = r / T; slot = r % T; loc_base = s * k * k;
+  }
   const int seq = step_seqs[s];
   const int n = seq_len[seq];
   int id;
@@ -63,8 +74,8 @@ __global__ void assemble_step_kernel(RowMeta m, const int32_t *__restrict__ step
       if (sampling) m.skey[r] = position_key(seed, seq, n + slot + 1);        // a causal slot predicts the next position
     } else {
       const int b = (slot - k) / k, i = (slot - k) % k;
-      m.pos[r] = n + b + 1 + i; m.nvis[r] = n + b + 1; m.loc0[r] = s * k * k + b * k; m.nloc[r] = k;
-      m.cache_pos[r] = -1; m.local_idx[r] = s * k * k + b * k + i;
+      m.pos[r] = n + b + 1 + i; m.nvis[r] = n + b + 1; m.loc0[r] = loc_base + b * k; m.nloc[r] = k;
+      m.cache_pos[r] = -1; m.local_idx[r] = loc_base + b * k + i;
       if (sampling) m.skey[r] = position_key(seed, seq, n + b + 1 + i);       // a mask slot predicts its own position
     }
   }
@@ -378,16 +389,17 @@ __global__ void slab_sum_kernel(const float *__restrict__ in, int S, size_t stri
 // ---------------------------------------------------------------------------
 __global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const int32_t *__restrict__ tgt_ids,
                                      const int32_t *__restrict__ step_seqs,
-                                     const int32_t *__restrict__ forced, int k, int n_blocks, int k_max,
+                                     const int32_t *__restrict__ forced, int k, int n_blocks, StepLayout lay, int k_max,
                                      int32_t *__restrict__ block_ids, int32_t *__restrict__ blk_len, int32_t *__restrict__ step_L,
                                      int32_t *__restrict__ out /*[n_seqs][k_max+1]*/, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
   const int s = blockIdx.x, lane = threadIdx.x;
+  if (lay.k) { k = lay.k[s]; n_blocks = k; }
   const int T = k * (n_blocks + 1);
   const int seq = step_seqs[s];
-  const int32_t *ids = arg_ids + (size_t)s * T;
+  const int32_t *ids = arg_ids + (lay.k ? (size_t)lay.off[s] : (size_t)s * T);
   int32_t *blk = block_ids + (size_t)seq * k_max;
   const int valid = blk_len[seq];
   const int tgt = lane < k ? (tgt_ids ? tgt_ids[(size_t)s * k + lane] : ids[lane]) : -1;
@@ -501,12 +513,13 @@ __global__ void prefill_finish_kernel(const int32_t *__restrict__ arg_ids, int r
 // by an exact zero, which must stay zero.)  Grid (n_seqs, n_layers).
 // ---------------------------------------------------------------------------
 __global__ void kv_commit_kernel(const int32_t *__restrict__ step_seqs, const int32_t *__restrict__ step_n,
-                                 const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, int poison,
-                                 KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride, TlSlot tl) {
+                                 const int32_t *__restrict__ step_L, int32_t *__restrict__ seq_len, int k, const int32_t *__restrict__ step_k,
+                                 int poison, KvGeom g, bf16 *__restrict__ kv_base, size_t pool_stride, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
   const int s = blockIdx.x, l = blockIdx.y;
+  if (step_k) k = step_k[s];
   const int seq = step_seqs[s];
   const int n = step_n[s], L = step_L[s];
   if (l == 0 && threadIdx.x == 0) seq_len[seq] = n + L;

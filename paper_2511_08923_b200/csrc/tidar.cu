@@ -49,6 +49,13 @@ struct tidar_ctx {
   bf16 *kv = nullptr;
   RowMeta meta{};
   int32_t *d_blk_len = nullptr;    // [max_batch]: drafts a sequence's block holds (the block length of its last pass)
+  // a step whose sequences use different block lengths: per listed sequence its k, first row, first local row;
+  // per query tile of the attention kernel its first row and the end of its sequence's rows
+  int32_t *d_step_k = nullptr, *d_step_off = nullptr, *d_step_loc = nullptr, *d_tile_row0 = nullptr, *d_tile_rend = nullptr;
+  int32_t *h_lay = nullptr;        // pinned staging for those five arrays
+  size_t lay_ints = 0;
+  int mixed_tiles = 0;             // query tiles of the current mixed step
+  std::vector<int> pending_ks;
   float *d_run_max = nullptr, *d_run_sum = nullptr, *d_tgt_logit = nullptr, *d_logprob = nullptr;   // likelihood scoring, per row
   int32_t *d_target = nullptr;
   std::vector<CUtensorMap> tm_lm_chunks;   // the LM head in vocabulary chunks of lm_chunk rows (scoring)
@@ -167,6 +174,11 @@ void layout(tidar_ctx &x, void *arena, size_t *bytes) {
   x.meta.skey = cv.take<uint32_t>(R);
   x.d_seq_len = cv.take<int32_t>(c.max_batch);
   x.d_blk_len = cv.take<int32_t>(c.max_batch);
+  // one block, so that one copy brings the whole layout of a mixed step over (same order in h_lay)
+  x.lay_ints = 3 * (size_t)(c.max_batch + 1) + 2 * (size_t)(x.R_head + c.max_batch);
+  x.d_step_k = cv.take<int32_t>(x.lay_ints);
+  x.d_step_off = x.d_step_k + (c.max_batch + 1); x.d_step_loc = x.d_step_off + (c.max_batch + 1);
+  x.d_tile_row0 = x.d_step_loc + (c.max_batch + 1); x.d_tile_rend = x.d_tile_row0 + (x.R_head + c.max_batch);
   x.d_run_max = cv.take<float>(R); x.d_run_sum = cv.take<float>(R); x.d_tgt_logit = cv.take<float>(R); x.d_logprob = cv.take<float>(R);
   x.d_target = cv.take<int32_t>(R);
   x.d_block = cv.take<int32_t>((size_t)c.max_batch * c.k_max);
@@ -432,7 +444,8 @@ int attn_key_splits(const tidar_ctx *c, int units, int key_tiles_hint) {
 
 struct AttnMaps { const CUtensorMap *q, *k, *v, *kloc, *vloc; int page_base_k, page_base_v; };
 
-// rows_per_group: slots per sequence (k(k+1) in a step; all rows in a first-pass chunk).
+// rows_per_group: slots per sequence (k(k+1) in a step; all rows in a first-pass chunk); <= 0: the
+// sequences' groups differ in size and the query tiles come from the mixed step's tile table.
 // key_tiles_hint: rough number of 64-key tiles per row, to size the key split.
 void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 *O, int R, int rows_per_group, int key_tiles_hint) {
   const tidar_config &cf = c->cfg;
@@ -440,9 +453,15 @@ void launch_attention_tc(tidar_ctx *c, const AttnMaps &m, const KvGeom &g, bf16 
   a.R = R; a.rows_per_group = rows_per_group;
   a.G = cf.n_q_heads / cf.n_kv_heads; a.Hq = cf.n_q_heads; a.Hkv = cf.n_kv_heads;
   a.spt = 128 / a.G;
-  a.tiles_per_group = (rows_per_group + a.spt - 1) / a.spt;
-  a.n_groups = (R + rows_per_group - 1) / rows_per_group;
-  const int units = a.n_groups * a.tiles_per_group * a.Hkv;
+  if (rows_per_group > 0) {
+    a.tiles_per_group = (rows_per_group + a.spt - 1) / a.spt;
+    a.n_groups = (R + rows_per_group - 1) / rows_per_group;
+    a.n_tiles = a.n_groups * a.tiles_per_group;
+  } else {                       // groups of different sizes: the tile table of the mixed step
+    a.rows_per_group = R; a.tiles_per_group = 1; a.n_groups = 1;
+    a.tile_row0 = c->d_tile_row0; a.tile_rend = c->d_tile_rend; a.n_tiles = c->mixed_tiles;
+  }
+  const int units = a.n_tiles * a.Hkv;
   a.splits = attn_key_splits(c, units, key_tiles_hint);
   a.seq = c->meta.seq; a.nvis = c->meta.nvis; a.loc0 = c->meta.loc0; a.nloc = c->meta.nloc;
   a.page_table = g.page_table; a.pages_per_seq = g.pages_per_seq;
@@ -672,10 +691,16 @@ int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
 
 // Enqueues every operation of one decode step for the sequences staged in h_stage.
 // k: block length of this step; ar: plain autoregressive step (the causal section alone).
-int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar) {
+// mixed_R > 0: the listed sequences use different block lengths (layout staged in h_lay, mixed_R rows in all).
+int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, int mixed_R = 0) {
   const tidar_config &cf = c->cfg;
   const int n_blocks = ar ? 0 : k;
-  const int T = k * (n_blocks + 1), R = n_seqs * T;
+  const int T = k * (n_blocks + 1), R = mixed_R > 0 ? mixed_R : n_seqs * T;
+  StepLayout lay{nullptr, nullptr, nullptr, n_seqs};
+  if (mixed_R > 0) {
+    CUDA_TRY(c, cudaMemcpyAsync(c->d_step_k, c->h_lay, c->lay_ints * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    lay.k = c->d_step_k; lay.off = c->d_step_off; lay.loc = c->d_step_loc;
+  }
   if (c->timeline) {
     c->tl_n = 0; c->tl_cls.clear();
     CUDA_TRY(c, cudaMemsetAsync(c->d_tl, 0, 2 * tidar_ctx::TL_MAX * sizeof(unsigned long long), c->stream));
@@ -684,21 +709,21 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar) {
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
-    launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, c->d_blk_len, k, n_blocks, cf.k_max,
+    launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, c->d_blk_len, k, n_blocks, lay, cf.k_max,
                cf.mask_token_id, c->d_step_n, c->embed, cf.d_model, c->X, cf.temperature > 0.f ? 1 : 0, (unsigned long long)cf.sample_seed, l.tl);
   }
   // beta < 1: the verified prediction of causal slot j mixes its row with the first slot of block j
   MixRows mix;
   if (cf.beta < 1.0f && !ar) { mix.n = n_seqs * k; mix.k = k; mix.a0 = 0; mix.a_seq = T; mix.a_j = 1; mix.b0 = k; mix.b_seq = T; mix.b_j = k; }
-  if (int rc = forward_rows(c, R, true, T, key_tiles_hint, mix)) return rc;
+  if (int rc = forward_rows(c, R, true, mixed_R > 0 ? 0 : T, key_tiles_hint, mix)) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
     launch_after(verify_select_kernel, n_seqs, 32, 0, c->stream, c->d_arg_idx, mix.n ? c->d_arg_idx + R : (const int32_t *)nullptr, c->d_step_seqs,
-               c->d_forced, k, n_blocks, cf.k_max, c->d_block, c->d_blk_len, c->d_step_L, c->d_out, l.tl);
+               c->d_forced, k, n_blocks, lay, cf.k_max, c->d_block, c->d_blk_len, c->d_step_L, c->d_out, l.tl);
   }
   {
     Launch l(c, TIDAR_TC_VERIFY);
-    launch_after(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k,
+    launch_after(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k, lay.k,
                (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride, l.tl);
   }
   CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
@@ -775,11 +800,61 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   if (!launched)
     if (int rc = record_step(c, n_seqs, k, hint, ar)) return rc;
   c->pending_k = k;
+  c->pending_ks.clear();
   c->pending_seqs.assign(seqs, seqs + n_seqs);
   c->pending = true;
   c->last_hidden_off = 0;
   c->last_rows = R + ((cf.beta < 1.0f && !ar) ? n_seqs * k : 0); c->last_first_pos = -1;      // the mixed rows follow the slots
   // the host tracks lengths without reading the device when L is forced
+  return TIDAR_OK;
+}
+
+// A step in which listed sequence i uses block length ks[i] (Section 5: the block length follows the
+// compute profile; nothing in the method ties the sequences of a batch to one length).  Equal lengths
+// take the ordinary path (and its captured graph); different lengths run as plain launches over
+// R = sum k_i (k_i + 1) rows with a per-sequence row layout and an attention tile table.
+int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *ks, const int32_t *forced) {
+  const tidar_config &cf = c->cfg;
+  if (!seqs || !ks || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
+  bool same = true;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (ks[i] < 1 || ks[i] > cf.k_max) return fail(c, TIDAR_EINVAL, "block length %d of entry %d outside [1, k_max = %d]", ks[i], i, cf.k_max);
+    same = same && ks[i] == ks[0];
+  }
+  if (same) return enqueue_step(c, seqs, n_seqs, forced, false, ks[0], false);
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is already in flight; call tidar_step_wait first");
+  if (cf.beta < 1.0f) return fail(c, TIDAR_EINVAL, "beta < 1 needs one block length for all sequences of a step");
+  for (int i = 0; i < n_seqs; ++i) {
+    const int q = seqs[i], k = ks[i];
+    if (q < 0 || q >= cf.max_batch || !c->seqs[q].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", q);
+    for (int j = 0; j < i; ++j) if (seqs[j] == q) return fail(c, TIDAR_EINVAL, "sequence %d listed twice", q);
+    const int f = forced ? forced[i] : 0;
+    if (f < 0 || f > k) return fail(c, TIDAR_EINVAL, "forced acceptance %d outside [0, %d]", f, k);
+    if (c->seqs[q].n + 2 * k > cf.max_seq_len)
+      return fail(c, TIDAR_ECAPACITY, "sequence %d: n + 2k = %d exceeds max_seq_len %d", q, c->seqs[q].n + 2 * k, cf.max_seq_len);
+  }
+  for (int i = 0; i < n_seqs; ++i)
+    if (int rc = ensure_pages(c, seqs[i], c->seqs[seqs[i]].n + ks[i])) return rc;
+  const int mb = cf.max_batch, spt = 128 / (cf.n_q_heads / cf.n_kv_heads);
+  int32_t *hk = c->h_lay, *hoff = hk + (mb + 1), *hloc = hoff + (mb + 1), *ht0 = hloc + (mb + 1), *hte = ht0 + (c->R_head + mb);
+  int R = 0, loc = 0, tiles = 0, min_nk = 1 << 30;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int k = ks[i], T = k * (k + 1);
+    hk[i] = k; hoff[i] = R; hloc[i] = loc;
+    for (int r0 = R; r0 < R + T; r0 += spt) { ht0[tiles] = r0; hte[tiles] = R + T; ++tiles; }
+    R += T; loc += k * k;
+    min_nk = std::min(min_nk, c->seqs[seqs[i]].n + k);
+    c->h_stage[i] = seqs[i]; c->h_stage[mb + i] = forced ? forced[i] : 0;
+  }
+  hk[n_seqs] = 0; hoff[n_seqs] = R; hloc[n_seqs] = loc;
+  c->mixed_tiles = tiles;
+  if (int rc = record_step(c, n_seqs, ks[0], (min_nk + 63) / 64, false, R)) return rc;
+  c->pending_k = 0;
+  c->pending_ks.assign(ks, ks + n_seqs);
+  c->pending_seqs.assign(seqs, seqs + n_seqs);
+  c->pending = true;
+  c->last_hidden_off = 0;
+  c->last_rows = R; c->last_first_pos = -1;
   return TIDAR_OK;
 }
 
@@ -802,7 +877,7 @@ int finish_step(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
   for (size_t i = 0; i < c->pending_seqs.size(); ++i) {
     const int L = c->h_pinned[i * (km + 1)];
     c->seqs[c->pending_seqs[i]].n += L;
-    c->seqs[c->pending_seqs[i]].k = c->pending_k;        // the block the step left has this many entries
+    c->seqs[c->pending_seqs[i]].k = c->pending_ks.empty() ? c->pending_k : c->pending_ks[i];   // entries of the block the step left
     if (out_n) out_n[i] = L;
     if (out_tokens) for (int j = 0; j < km; ++j) out_tokens[i * km + j] = j < L ? c->h_pinned[i * (km + 1) + 1 + j] : -1;
   }
@@ -866,10 +941,11 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
   for (int i = 0; i < c->n_pages; ++i) c->free_pages[i] = i;
   uint32_t st = 0x9e3779b9u;
   for (int i = c->n_pages - 1; i > 0; --i) { st = st * 1664525u + 1013904223u; std::swap(c->free_pages[i], c->free_pages[(st >> 8) % (i + 1)]); }
-  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch + 16) * sizeof(int), cudaHostAllocDefault);
+  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch + 16 + c->lay_ints) * sizeof(int), cudaHostAllocDefault);
   if (e != cudaSuccess) { delete c; return fail(nullptr, TIDAR_ECUDA, "cudaHostAlloc: %s", cudaGetErrorString(e)); }
   c->h_stage = c->h_pinned + (size_t)cfg->max_batch * (cfg->k_max + 1);
   c->h_status = c->h_stage + 2 * cfg->max_batch;
+  c->h_lay = c->h_status + 16;
   c->h_status[0] = 0;
   e = cudaMemsetAsync(c->d_seq_len, 0, cfg->max_batch * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 64 * sizeof(int), c->stream);
@@ -953,6 +1029,12 @@ int tidar_step_k(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t k, c
   if (!c) return TIDAR_EINVAL;
   if (k < 1) return fail(c, TIDAR_EINVAL, "block length must be at least 1");
   if (int rc = enqueue_step(c, seqs, n_seqs, forced, false, k, false)) return rc;
+  return finish_step(c, out_tokens, out_n);
+}
+
+int tidar_step_ks(tidar_ctx *c, const int32_t *seqs, int32_t n_seqs, const int32_t *ks, const int32_t *forced, int32_t *out_tokens, int32_t *out_n) {
+  if (!c) return TIDAR_EINVAL;
+  if (int rc = enqueue_step_mixed(c, seqs, n_seqs, ks, forced)) return rc;
   return finish_step(c, out_tokens, out_n);
 }
 

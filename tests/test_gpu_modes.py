@@ -121,6 +121,90 @@ def test_block_length_chosen_per_step(tiny, impl):
     _close(t)
 
 
+@pytest.mark.parametrize("impl", IMPLS)
+def test_block_length_per_sequence_within_one_step(tiny, impl):
+    """tidar_step_ks: three sequences with block lengths 2, 4 and 3 share one pass (20 + 6 + 12 slots laid
+    out sequence after sequence).  Per sequence the logits, the acceptance and the committed cache are
+    those of the oracle's own step with that sequence's block length."""
+    from paper_2511_08923_b200 import TidarError, bf16_bits_to_f32
+    sh, wt, cfg, w, prompt = tiny
+    ks = [4, 2, 3]
+    prompts = [prompt, prompt_ids(sh, n=sh.prompt_len - 5, seed=sh.seed + 1), prompt_ids(sh, n=sh.prompt_len + 9, seed=sh.seed + 2)]
+    t = _gpu(sh, wt, impl, k_max=4, debug=1, max_batch=3, max_seq_len=256)
+    states = []
+    for q, (p, k) in enumerate(zip(prompts, ks)):
+        t.prefill(q, p, k)
+        states.append(O.prefill(cfg, w, p, k)[0])
+    order = [2, 0, 1]                                              # listed order need not be slot order
+    for step in range(5):
+        forced = [0, 0, 0] if step != 2 else [1, 2, 1]
+        blocks, outs = [], []
+        for q in order:
+            t.set_block(q, states[q].block)                        # teacher-forced: the caches stay comparable
+            blocks.append(states[q].block.copy())
+        for i, q in enumerate(order):
+            outs.append(O.step(cfg, w, states[q], forced=forced[i]))
+        toks, L = t.step_ks(order, [ks[q] for q in order], forced if step == 2 else None)
+        n_rows, _ = t.last_rows()
+        assert n_rows == sum(ks[q] * (ks[q] + 1) for q in order)
+        lg = t.logits(0, n_rows)
+        ids = t.argmax(0, n_rows)
+        r0 = 0
+        for i, q in enumerate(order):
+            k = ks[q]; T = k * (k + 1)
+            assert np.abs(lg[r0:r0 + T] - outs[i].fwd.logits).max() <= TOL_LOGITS, (step, q)
+            L_ref = O.accept_length(blocks[i], ids[r0:r0 + k], forced[i])
+            assert L[i] == L_ref
+            assert toks[i] == [int(x) for x in blocks[i][1:L_ref]] + [int(ids[r0 + L_ref - 1])]
+            if L[i] != outs[i].L or toks[i] != outs[i].emitted:    # only a near-tie may be decided the other way
+                assert top1_margin(outs[i].fwd.logits[:k]).min() <= MARGIN, (step, q, L[i], outs[i].L)
+                pytest.skip("near-tie in a verified position of the synthetic model")
+            assert t.seq_len(q) == states[q].n
+            assert t.get_block(q, k)[0] == int(states[q].block[0])
+            r0 += T
+    for q in range(3):
+        n = t.seq_len(q)
+        for l in range(cfg.n_layers):
+            K, V = t.kv(q, l, 0, n)
+            check_rows(bf16_bits_to_f32(K).reshape(n, -1), states[q].k_cache[l].reshape(n, -1), f"K seq {q} layer {l}")
+            check_rows(bf16_bits_to_f32(V).reshape(n, -1), states[q].v_cache[l].reshape(n, -1), f"V seq {q} layer {l}")
+    with pytest.raises(TidarError):
+        t.step_ks([0, 1], [4, 5])                                  # above k_max
+    with pytest.raises(TidarError):
+        t.step_ks([0, 1], [2, 3], [3, 1])                          # forced acceptance above that sequence's length
+    toks, L = t.step_ks([0, 1, 2], [3, 3, 3])                      # equal lengths: the ordinary step
+    assert all(1 <= x <= 3 for x in L)
+    _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_mixed_block_lengths_keep_the_autoregressive_continuation(tiny, impl):
+    """With beta = 1 and greedy decoding every sequence of a mixed step still emits the model's
+    autoregressive continuation, whatever lengths the steps choose (changing from step to step)."""
+    sh, wt, cfg, w, prompt = tiny
+    n_new = 28
+    prompts = [prompt, prompt_ids(sh, n=sh.prompt_len + 3, seed=sh.seed + 7)]
+    refs, upto = [], []
+    for p in prompts:
+        ar = O.ar_generate(cfg, w, p, n_new + 8)
+        m = top1_margin(O.causal_forward(cfg, w, list(p) + ar).logits[len(p) - 1:len(p) - 1 + n_new])
+        unsure = np.nonzero(m <= MARGIN)[0]
+        refs.append(ar); upto.append(int(unsure[0]) if len(unsure) else n_new)
+    t = _gpu(sh, wt, impl, k_max=8, max_batch=2, max_seq_len=256)
+    out = [[t.prefill(q, p, 4)] for q, p in enumerate(prompts)]
+    plan = [(2, 8), (8, 3), (5, 5), (1, 7), (8, 8), (3, 6), (6, 2), (8, 4), (4, 8), (7, 7), (8, 8), (8, 8)]
+    for ka, kb in plan:
+        toks, L = t.step_ks([0, 1], [ka, kb])
+        for q in range(2):
+            out[q].extend(toks[q])
+            assert t.seq_len(q) == len(prompts[q]) + len(out[q]) - 1
+        if min(len(o) for o in out) >= n_new:
+            break
+    for q in range(2):
+        assert out[q][:upto[q]] == refs[q][:upto[q]], q
+    _close(t)
+
+
 # ---- beta < 1 ------------------------------------------------------------------------------------
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("beta", [0.0, 0.5])
