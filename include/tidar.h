@@ -177,8 +177,8 @@ int tidar_step_k(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t 
  * the method ties the sequences of a batch to one length.  The pass has sum_i ks[i]*(ks[i]+1) token
  * slots, sequence after sequence.  Per sequence the results are those of tidar_step_k with that
  * sequence's length (same tokens; hidden states up to the rounding of a different row count).
- * forced_accept[i] in [0, ks[i]].  Equal lengths take tidar_step_k's path; different lengths are
- * launched kernel by kernel (no captured graph) and need beta == 1 (TIDAR_EINVAL otherwise).
+ * forced_accept[i] in [0, ks[i]].  Equal lengths take tidar_step_k's path; different lengths need
+ * beta == 1 (TIDAR_EINVAL otherwise).
  * out_tokens / out_n as in tidar_step.                                                        */
 int tidar_step_ks(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs, const int32_t *ks /*host,[n_seqs]*/,
                   const int32_t *forced_accept /*host or NULL*/, int32_t *out_tokens /*host,[n_seqs][k_max]*/,
@@ -189,6 +189,24 @@ int tidar_step_ks(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t
  * selects 288, one row block of the projection kernels, about where the 8B-class step
  * leaves the memory-bound region on a B200 (measured ridge: 220 .. 288 rows).  Host only. */
 int tidar_ridge_k(const tidar_ctx *ctx, int32_t n_seqs, int32_t row_budget);
+
+/* Block lengths for one step of a batch under a budget of token slots (paper Section 5: the extra
+ * slots are free only while the pass stays memory-bound, and a scheduler should spend them where they
+ * can yield tokens).  want[i] (host, [n_seqs], or NULL) caps the block of sequence i, e.g. at the number
+ * of tokens it still has to produce; out_ks[i] (host, [n_seqs]) receives a length in
+ * [1, min(k_max, want[i])].  The plan maximises sum_i out_ks[i] subject to
+ * sum_i out_ks[i]*(out_ks[i]+1) <= row_budget by always lengthening the shortest block that may still
+ * grow (one more draft at length k costs 2(k+1) slots); when even length 1 everywhere exceeds the
+ * budget every sequence gets 1.  row_budget <= 0 selects 288 as in tidar_ridge_k.  Feed the result to
+ * tidar_step_ks.  Host only, needs no context or device.  TIDAR_EINVAL for a non-positive n_seqs,
+ * k_max or want[i], or a null out_ks.                                                          */
+int tidar_plan_ks(int32_t n_seqs, int32_t k_max, int32_t row_budget, const int32_t *want /*host or NULL*/, int32_t *out_ks /*host*/);
+
+/* Returns a sequence slot's KV pages to the pool and marks it not prefilled, so that another prompt
+ * can take the slot (sequences of a batch finish at different times; a step lists any subset of the
+ * prefilled slots).  A slot that holds nothing is left as it is.  TIDAR_EINVAL while a step is in
+ * flight or for a slot outside [0, max_batch).                                                   */
+int tidar_release(tidar_ctx *ctx, int32_t seq);
 
 /* One plain autoregressive step (paper Section 3.1: the model keeps a causal, chain-factorised
  * mode): a single causal slot per sequence, the settled token at position n, no mask slots.

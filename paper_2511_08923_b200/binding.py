@@ -67,6 +67,8 @@ def load(rebuild: bool = False) -> C.CDLL:
         "tidar_step_wait": (C.c_int, [ctxp, P(I32), P(I32)]),
         "tidar_step_k": (C.c_int, [ctxp, P(I32), I32, I32, P(I32), P(I32), P(I32)]),
         "tidar_step_ks": (C.c_int, [ctxp, P(I32), I32, P(I32), P(I32), P(I32), P(I32)]),
+        "tidar_plan_ks": (C.c_int, [I32, I32, I32, P(I32), P(I32)]),
+        "tidar_release": (C.c_int, [ctxp, I32]),
         "tidar_ar_step": (C.c_int, [ctxp, P(I32), I32, P(I32)]),
         "tidar_ridge_k": (C.c_int, [ctxp, I32, I32]),
         "tidar_score": (C.c_int, [ctxp, I32, P(I32), I32, P(C.c_float)]),
@@ -244,6 +246,10 @@ class Tidar:
         self._check(self.lib.tidar_step_ks(self.ctx, _ip(s), len(s), _ip(kk), _ip(f) if f is not None else None, _ip(toks), _ip(n)))
         return [toks[i, :n[i]].tolist() for i in range(len(s))], n.tolist()
 
+    def release(self, seq: int):
+        """Gives a sequence slot's KV pages back (see tidar_release)."""
+        self._check(self.lib.tidar_release(self.ctx, seq))
+
     def ar_step(self, seqs: Sequence[int]) -> List[int]:
         """One plain autoregressive step: one new token per sequence (see tidar_ar_step)."""
         s = _i32(seqs)
@@ -367,6 +373,19 @@ class Tidar:
         self._check(self.lib.tidar_attention(
             self.ctx, q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), k_pages.shape[0], page_table.data_ptr(), page_table.shape[1],
             seq_len.data_ptr(), k_local.data_ptr(), v_local.data_ptr(), out.data_ptr(), n_seqs, k))
+
+
+def plan_ks(n_seqs: int, k_max: int, row_budget: int = 0, want: Optional[Sequence[int]] = None) -> List[int]:
+    """Block lengths for one step of a batch under a budget of token slots (see tidar_plan_ks)."""
+    lib = load()
+    w = _i32(want) if want is not None else None
+    if w is not None and len(w) != n_seqs:
+        raise ValueError("one cap per sequence")
+    out = np.empty(max(n_seqs, 1), dtype=np.int32)
+    rc = lib.tidar_plan_ks(n_seqs, k_max, row_budget, _ip(w) if w is not None else None, _ip(out))
+    if rc != 0:
+        raise TidarError(rc, (lib.tidar_last_error(None) or b"").decode())
+    return out[:n_seqs].tolist()
 
 
 def attention_static(q, k_pages, v_pages, page_table, seq_len, k_local, v_local, out, n_seqs: int, k: int,

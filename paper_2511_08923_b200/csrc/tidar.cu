@@ -84,7 +84,7 @@ struct tidar_ctx {
   float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
   // the launches of one decode step as an executable graph, valid for one (k, n_seqs, attention split)
-  struct StepGraph { int k = 0, n_seqs = 0, splits = 0; bool ar = false, timeline = false; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
+  struct StepGraph { int k = 0, n_seqs = 0, splits = 0, mixed_R = 0, tiles = 0; bool ar = false, timeline = false; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
   bool graphs_ok = true;
   bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
@@ -732,6 +732,47 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, in
   return TIDAR_OK;
 }
 
+// Every launch of a step has the same arguments from step to step (lengths, page tables, token
+// blocks and, for a step of mixed block lengths, the row layout live in device memory), except
+// for the grid sizes and the attention key split, so the step is captured once per (k, n_seqs,
+// rows, query tiles, split) and replayed.  Per-launch timing and the debug read-backs use plain
+// launches.  tiles: query tiles of the attention kernel per KV head.
+int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles) {
+  const tidar_config &cf = c->cfg;
+  if (cf.impl == 0 && c->graphs_ok && !c->timing && !(cf.debug & (1 | 8))) {
+    const int splits = attn_key_splits(c, tiles * cf.n_kv_heads, hint);
+    tidar_ctx::StepGraph &sg = c->sg;
+    if (!sg.exec || sg.k != k || sg.ar != ar || sg.n_seqs != n_seqs || sg.splits != splits || sg.timeline != c->timeline ||
+        sg.mixed_R != mixed_R || sg.tiles != tiles) {
+      if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
+      const int64_t l0 = c->launches;
+      cudaGraph_t graph = nullptr;
+      int rc = TIDAR_OK;
+      cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
+      if (e == cudaSuccess) {
+        rc = record_step(c, n_seqs, k, hint, ar, mixed_R);
+        e = cudaStreamEndCapture(c->stream, &graph);
+      }
+      if (e == cudaSuccess && rc == TIDAR_OK && graph) e = cudaGraphInstantiate(&sg.exec, graph, 0);
+      if (graph) cudaGraphDestroy(graph);
+      if (e != cudaSuccess || rc != TIDAR_OK || !sg.exec) {
+        cudaGetLastError();                         // capture is not available here: plain launches from now on
+        sg.exec = nullptr; c->graphs_ok = false;
+      } else {
+        sg.k = k; sg.ar = ar; sg.n_seqs = n_seqs; sg.splits = splits; sg.timeline = c->timeline; sg.mixed_R = mixed_R; sg.tiles = tiles;
+        sg.launches = c->launches - l0;
+      }
+      c->launches = l0;
+    }
+    if (sg.exec) {
+      CUDA_TRY(c, cudaGraphLaunch(sg.exec, c->stream));
+      c->launches += sg.launches;
+      return TIDAR_OK;
+    }
+  }
+  return record_step(c, n_seqs, k, hint, ar, mixed_R);
+}
+
 // k_step: block length of this step (0 = the one the sequences' last pass left, which must then be
 // the same for all of them); ar: plain autoregressive step (k_step is 1).
 int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced, int k_step = 0, bool ar = false) {
@@ -762,43 +803,8 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
   int min_n = 1 << 30;
   for (int i = 0; i < n_seqs; ++i) min_n = std::min(min_n, c->seqs[seqs[i]].n);
   const int hint = (min_n + k + 63) / 64;
-  // Every launch of a step has the same arguments from step to step (lengths, page tables and
-  // token blocks live in device memory), except for the attention key split, so the step is
-  // captured once per (k, n_seqs, split) and replayed.  Per-launch timing and the debug
-  // read-backs use plain launches.
-  bool launched = false;
-  if (cf.impl == 0 && c->graphs_ok && !c->timing && !(cf.debug & (1 | 8))) {
-    const int G = cf.n_q_heads / cf.n_kv_heads, spt = 128 / G;
-    const int splits = attn_key_splits(c, n_seqs * ((T + spt - 1) / spt) * cf.n_kv_heads, hint);
-    tidar_ctx::StepGraph &sg = c->sg;
-    if (!sg.exec || sg.k != k || sg.ar != ar || sg.n_seqs != n_seqs || sg.splits != splits || sg.timeline != c->timeline) {
-      if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
-      const int64_t l0 = c->launches;
-      cudaGraph_t graph = nullptr;
-      int rc = TIDAR_OK;
-      cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
-      if (e == cudaSuccess) {
-        rc = record_step(c, n_seqs, k, hint, ar);
-        e = cudaStreamEndCapture(c->stream, &graph);
-      }
-      if (e == cudaSuccess && rc == TIDAR_OK && graph) e = cudaGraphInstantiate(&sg.exec, graph, 0);
-      if (graph) cudaGraphDestroy(graph);
-      if (e != cudaSuccess || rc != TIDAR_OK || !sg.exec) {
-        cudaGetLastError();                         // capture is not available here: plain launches from now on
-        sg.exec = nullptr; c->graphs_ok = false;
-      } else {
-        sg.k = k; sg.ar = ar; sg.n_seqs = n_seqs; sg.splits = splits; sg.timeline = c->timeline; sg.launches = c->launches - l0;
-      }
-      c->launches = l0;
-    }
-    if (sg.exec) {
-      CUDA_TRY(c, cudaGraphLaunch(sg.exec, c->stream));
-      c->launches += sg.launches;
-      launched = true;
-    }
-  }
-  if (!launched)
-    if (int rc = record_step(c, n_seqs, k, hint, ar)) return rc;
+  const int spt = 128 / (cf.n_q_heads / cf.n_kv_heads);          // slots per attention query tile
+  if (int rc = replay_or_record_step(c, n_seqs, k, hint, ar, 0, n_seqs * ((T + spt - 1) / spt))) return rc;
   c->pending_k = k;
   c->pending_ks.clear();
   c->pending_seqs.assign(seqs, seqs + n_seqs);
@@ -811,8 +817,9 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
 
 // A step in which listed sequence i uses block length ks[i] (Section 5: the block length follows the
 // compute profile; nothing in the method ties the sequences of a batch to one length).  Equal lengths
-// take the ordinary path (and its captured graph); different lengths run as plain launches over
-// R = sum k_i (k_i + 1) rows with a per-sequence row layout and an attention tile table.
+// take the ordinary path; different lengths run over R = sum k_i (k_i + 1) rows with a per-sequence
+// row layout and an attention tile table (one captured graph serves every step with the same
+// number of sequences, rows and query tiles).
 int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *ks, const int32_t *forced) {
   const tidar_config &cf = c->cfg;
   if (!seqs || !ks || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
@@ -848,7 +855,8 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
   }
   hk[n_seqs] = 0; hoff[n_seqs] = R; hloc[n_seqs] = loc;
   c->mixed_tiles = tiles;
-  if (int rc = record_step(c, n_seqs, ks[0], (min_nk + 63) / 64, false, R)) return rc;
+  // a mixed step's kernels take every per-sequence length from the staged layout: the nominal k is unused
+  if (int rc = replay_or_record_step(c, n_seqs, 0, (min_nk + 63) / 64, false, R, tiles)) return rc;
   c->pending_k = 0;
   c->pending_ks.assign(ks, ks + n_seqs);
   c->pending_seqs.assign(seqs, seqs + n_seqs);
@@ -1053,6 +1061,37 @@ int tidar_ridge_k(const tidar_ctx *c, int32_t n_seqs, int32_t row_budget) {
   int k = 1;
   while (k < c->cfg.k_max && (long long)n_seqs * (k + 1) * (k + 2) <= row_budget) ++k;
   return k;
+}
+
+int tidar_plan_ks(int32_t n_seqs, int32_t k_max, int32_t row_budget, const int32_t *want, int32_t *out_ks) {
+  if (n_seqs < 1 || k_max < 1 || !out_ks) return fail(nullptr, TIDAR_EINVAL, "tidar_plan_ks: n_seqs and k_max must be positive, out_ks non-null");
+  if (row_budget <= 0) row_budget = 288;
+  long long rows = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (want && want[i] < 1) return fail(nullptr, TIDAR_EINVAL, "tidar_plan_ks: want[%d] = %d, must be at least 1", i, want[i]);
+    out_ks[i] = 1; rows += 2;
+  }
+  // One more draft for a sequence at length k costs 2(k + 1) rows and can yield one more token: the cost
+  // grows with k, so the shortest block that may still grow is always the best place for the next rows.
+  for (;;) {
+    int best = -1;
+    for (int i = 0; i < n_seqs; ++i) {
+      const int cap = want ? std::min(k_max, want[i]) : k_max;
+      if (out_ks[i] < cap && (best < 0 || out_ks[i] < out_ks[best])) best = i;
+    }
+    if (best < 0 || rows + 2 * (out_ks[best] + 1) > row_budget) break;
+    rows += 2 * (out_ks[best] + 1);
+    out_ks[best]++;
+  }
+  return TIDAR_OK;
+}
+
+int tidar_release(tidar_ctx *c, int32_t seq) {
+  if (!c) return TIDAR_EINVAL;
+  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (seq < 0 || seq >= c->cfg.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
+  if (c->seqs[seq].active) release_sequence(c, seq);
+  return TIDAR_OK;
 }
 
 int tidar_score(tidar_ctx *c, int32_t seq, const int32_t *ids, int32_t n, float *logprobs) {

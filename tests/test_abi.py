@@ -3,6 +3,7 @@ import ctypes as C
 import os
 import re
 
+import numpy as np
 import pytest
 
 from paper_2511_08923_b200 import binding, build
@@ -64,3 +65,31 @@ def test_init_without_gpu_fails_loudly():
     ctx = C.c_void_p()
     rc = lib.tidar_init(C.byref(_cfg()), C.byref(w), C.c_void_p(256), C.c_size_t(1 << 30), None, C.byref(ctx))
     assert rc == -4 and b"no CUDA device" in lib.tidar_last_error(None)
+
+
+def test_block_length_plan_is_optimal_under_the_row_budget():
+    """tidar_plan_ks (host only) against brute force: among all length vectors within the caps whose
+    slots sum_i k_i (k_i + 1) fit the budget, the plan has the largest sum of lengths; infeasible budgets
+    give all ones; the plan never exceeds a cap."""
+    import itertools
+    from paper_2511_08923_b200 import TidarError, plan_ks
+    rng = np.random.default_rng(5)
+    for trial in range(60):
+        n = int(rng.integers(1, 5)); k_max = int(rng.integers(1, 7))
+        want = [int(x) for x in rng.integers(1, 9, size=n)] if trial % 2 else None
+        budget = int(rng.integers(1, 120))
+        ks = plan_ks(n, k_max, budget, want)
+        caps = [min(k_max, w) for w in want] if want else [k_max] * n
+        assert all(1 <= k <= c for k, c in zip(ks, caps))
+        feasible = [v for v in itertools.product(*[range(1, c + 1) for c in caps]) if sum(k * (k + 1) for k in v) <= budget]
+        if not feasible:
+            assert ks == [1] * n
+        else:
+            assert sum(k * (k + 1) for k in ks) <= budget
+            assert sum(ks) == max(sum(v) for v in feasible), (n, k_max, budget, want, ks)
+            assert max(ks) - min(k for k, c in zip(ks, caps) if k < c or k == max(ks)) <= 1      # blocks that may still grow stay level
+    assert plan_ks(1, 16) == [16] and plan_ks(8, 16) == [6] * 4 + [5] * 4 and plan_ks(32, 16) == [3] * 16 + [2] * 16      # the default budget of 288 slots, used in full
+    assert plan_ks(3, 16, 288, [2, 16, 16]) == [2, 11, 11]                                            # 6 + 132 + 132 = 270 <= 288 < 270 + 24
+    for bad in [(0, 4, 10, None), (2, 0, 10, None), (2, 4, 10, [1, 0])]:
+        with pytest.raises(TidarError):
+            plan_ks(*bad)

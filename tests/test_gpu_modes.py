@@ -205,6 +205,89 @@ def test_mixed_block_lengths_keep_the_autoregressive_continuation(tiny, impl):
     _close(t)
 
 
+def test_mixed_step_graph_replay_matches_plain_launches():
+    """A step of mixed block lengths replays one captured graph for every length vector with the same
+    row and tile count ((3, 4, 2) and (2, 3, 4) here, the layout living in device memory); the same
+    teacher-forced steps launched kernel by kernel give identical tokens and bit-identical cached K/V."""
+    from dataclasses import replace as _r
+    from tidar_synth import CONFIGS as CONFIGS_, gen_model_weights as gen_model_weights_
+    sh = _r(CONFIGS_["8b"].reduced(2), vocab=8192)
+    wt = gen_model_weights_(sh)
+    prompts = [prompt_ids(sh, n=150 + 37 * q, seed=sh.seed + q) for q in range(3)]
+    plan = [([3, 4, 2], [2, 1, 2]), ([2, 3, 4], [1, 3, 4]), ([3, 4, 2], [3, 2, 1]), ([4, 4, 4], [4, 1, 2]), ([4, 2, 3], [2, 2, 3])]
+    runs = {}
+    for tag, debug in (("graph", 0), ("plain", 8)):
+        t = _gpu(sh, wt, 0, k_max=4, debug=debug, max_batch=3, max_seq_len=512)
+        rec = [t.prefill(q, p, 4) for q, p in enumerate(prompts)]
+        blocks = [[t.get_block(q, 4) for q in range(3)]]
+        l0 = t.launch_count()
+        for i, (ks, forced) in enumerate(plan):
+            if tag == "plain":
+                for q in range(3):
+                    t.set_block(q, runs["graph"]["blocks"][i][q])
+            rec.append(t.step_ks([0, 1, 2], ks, forced))
+            blocks.append([t.get_block(q, ks[q]) + [0] * (4 - ks[q]) for q in range(3)])
+        kv = [[t.kv(q, l, 0, t.seq_len(q)) for l in range(sh.n_layers)] for q in range(3)]
+        runs[tag] = {"rec": rec, "blocks": blocks, "kv": kv, "launches": t.launch_count() - l0}
+        _close(t)
+    assert runs["graph"]["rec"] == runs["plain"]["rec"]
+    assert runs["graph"]["blocks"] == runs["plain"]["blocks"]
+    assert runs["graph"]["launches"] == runs["plain"]["launches"]              # replayed launches are counted like recorded ones
+    for q in range(3):
+        for (k0, v0), (k1, v1) in zip(runs["graph"]["kv"][q], runs["plain"]["kv"][q]):
+            np.testing.assert_array_equal(k0, k1); np.testing.assert_array_equal(v0, v1)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_continuous_batching_with_planned_block_lengths(tiny, impl):
+    """Sequences that want different numbers of tokens share steps whose block lengths come from
+    tidar_plan_ks under a small slot budget; a finished sequence is released and the next prompt takes its
+    slot.  Every request still receives exactly the model's greedy autoregressive continuation."""
+    from paper_2511_08923_b200 import plan_ks
+    sh, wt, cfg, w, prompt = tiny
+    wants = [9, 21, 5, 14, 12]
+    prompts = [prompt_ids(sh, n=sh.prompt_len - 7 + 3 * r, seed=sh.seed + 11 + r) for r in range(len(wants))]
+    refs, sure = [], []
+    for p, n_new in zip(prompts, wants):
+        ar = O.ar_generate(cfg, w, p, n_new + 1)
+        m = top1_margin(O.causal_forward(cfg, w, list(p) + ar).logits[len(p) - 1:len(p) - 1 + n_new])
+        unsure = np.nonzero(m <= MARGIN)[0]
+        refs.append(ar[:n_new]); sure.append(int(unsure[0]) if len(unsure) else n_new)
+    k_max, budget = 6, 44
+    t = _gpu(sh, wt, impl, k_max=k_max, max_batch=2, max_seq_len=256)
+    waiting = list(range(len(wants)))
+    slot_req = {}                                   # slot -> request
+    out = {r: [] for r in range(len(wants))}
+    steps = 0
+    while waiting or slot_req:
+        for slot in range(2):                       # admit
+            if slot not in slot_req and waiting:
+                r = waiting.pop(0)
+                out[r].append(t.prefill(slot, prompts[r], 1))
+                slot_req[slot] = r
+        slots = sorted(s for s in slot_req if len(out[slot_req[s]]) < wants[slot_req[s]])
+        if slots:
+            remaining = [wants[slot_req[s]] - len(out[slot_req[s]]) for s in slots]
+            ks = plan_ks(len(slots), k_max, budget, remaining)
+            assert sum(k * (k + 1) for k in ks) <= budget and all(k <= rem for k, rem in zip(ks, remaining))
+            toks, L = t.step_ks(slots, ks)
+            for s, tk in zip(slots, toks):
+                out[slot_req[s]].extend(tk)
+            steps += 1
+        for s in list(slot_req):                    # retire
+            r = slot_req[s]
+            if len(out[r]) >= wants[r]:
+                assert len(out[r]) == wants[r]      # the cap keeps a step from running past the request
+                t.release(s)
+                del slot_req[s]
+        assert steps < 200
+    for r in range(len(wants)):
+        assert out[r][:sure[r]] == refs[r][:sure[r]], r
+    with pytest.raises(Exception):
+        t.step([0])                                 # released slots hold nothing
+    _close(t)
+
+
 # ---- beta < 1 ------------------------------------------------------------------------------------
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("beta", [0.0, 0.5])
