@@ -362,6 +362,7 @@ int gemm_tc_launch(tidar_ctx *c, int mode, const bf16 *A, int a_rows, const CUte
     a.inv_temp = c->cfg.temperature > 0.f ? 1.0f / c->cfg.temperature : 0.f; a.skey = c->meta.skey + c->head_row0;
   }
   a.status = c->d_status;
+  a.warm_epilogue = mode == gemm_tc::MODE_SWIGLU ? 1 : 0;
   const CUtensorMap *tmA = act_map(c, A, a_rows, K, a.box_rows);
   if (!tmA) return fail(c, TIDAR_ECUDA, "cuTensorMapEncodeTiled failed for an activation matrix (%d x %d, box %d)", a_rows, K, a.box_rows);
   const int items = a.total_items();
