@@ -12,12 +12,15 @@
 // Tiling: the G = Hq/Hkv query heads that share a KV head are packed into one 128-row
 // MMA tile (floor(128/G) slots x G heads), so K/V are read once per KV head.  Per key
 // tile: S = Q K^T (M 128, N 64, K hd) into TMEM (double buffered); the softmax warps read S
-// (one thread per row), keep a reference max and the running sum, write P (bf16) to shared
-// memory in the MMA operand layout; O += P V (M 128, N hd, K 64, V as the MN-major operand)
-// accumulates in TMEM over all key tiles.  The reference max is only raised when a tile
+// (one thread per row), keep a reference max and the running sum, and write P (bf16, two keys per
+// 32-bit column) back into the first half of the S buffer it came from; O += P V (M 128, N hd,
+// K 64, P as the tensor-memory operand, V as the MN-major shared-memory operand) accumulates in
+// TMEM over all key tiles.  P never touches shared memory: with P staged there the kernel moved
+// 128 KB through shared memory per key tile (Q 32 and K 16 read by Q K^T, P 16 written and read,
+// V 16, and the 32 KB the TMA writes), 1000 cycles at 128 B per cycle against 512 cycles of MMAs.  The reference max is only raised when a tile
 // exceeds it by more than 2^8 (P stays <= 256, exact enough in bf16/fp32); raising it
 // rescales the rows of O in TMEM, which happens in the first tiles only.  The CTA needs
-// <= 113 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
+// <= 97 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
 // share an SM and fill each other's dependency stalls.  The key range of a query tile can be
 // split over several CTAs; partial (max, sum, O) results are merged by attn_combine_kernel.
 #pragma once
@@ -27,7 +30,7 @@
 namespace attn_tc {
 
 constexpr int KT = 64;               // keys per tile (= page size)
-constexpr int KV_STAGES = 2;
+constexpr int K_STAGES = 3, V_STAGES = 2;   // K runs a tile further ahead: Q K^T of tile i + 1 is issued before P V of tile i
 constexpr int THREADS = 192;         // warp 0: TMA, warp 1: MMA, warps 2..5: softmax
 constexpr int MAX_SPLITS = 8;
 constexpr float RAISE_THRESHOLD = 8.f;   // log2 units
@@ -62,18 +65,16 @@ struct Smem {
   static constexpr int NH = HD / 64;                 // 64-element halves of a head
   static constexpr int Q_BYTES = 128 * HD * 2;
   static constexpr int KV_BYTES = KT * HD * 2;
-  static constexpr int P_BYTES = 128 * KT * 2;
   static constexpr int Q_OFF = 0;
   static constexpr int K_OFF = Q_OFF + Q_BYTES;
-  static constexpr int V_OFF = K_OFF + KV_STAGES * KV_BYTES;
-  static constexpr int P_OFF = V_OFF + KV_STAGES * KV_BYTES;
-  static constexpr int BAR_OFF = P_OFF + P_BYTES;    // mbarriers and a few words
+  static constexpr int V_OFF = K_OFF + K_STAGES * KV_BYTES;
+  static constexpr int BAR_OFF = V_OFF + V_STAGES * KV_BYTES;    // mbarriers and a few words
   static constexpr int TOTAL = BAR_OFF + 256;
   static constexpr int TMEM_COLS = 256;              // 2 x 64 (S) + HD (O) <= 256
 };
 
 struct Ctl {                                         // lives at Smem::BAR_OFF
-  uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES], s_full[2], s_empty[2], p_full, p_empty;
+  uint64_t q_full, k_full[K_STAGES], k_empty[K_STAGES], v_full[V_STAGES], v_empty[V_STAGES], s_full[2], s_empty[2], p_full[2];
   uint32_t tmem_base;
   int abort_flag, max_nvis, loc_lo, loc_hi;
 };
@@ -111,12 +112,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   if (threadIdx.x == 0) {
     ctl.abort_flag = 0; ctl.max_nvis = 0; ctl.loc_lo = 0x7fffffff; ctl.loc_hi = 0;
     sm100::mbar_init(sm100::smem_u32(&ctl.q_full), 1);
-    for (int s = 0; s < KV_STAGES; ++s) {
-      sm100::mbar_init(sm100::smem_u32(&ctl.k_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.k_empty[s]), 1);
-      sm100::mbar_init(sm100::smem_u32(&ctl.v_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.v_empty[s]), 1);
-    }
-    for (int b = 0; b < 2; ++b) { sm100::mbar_init(sm100::smem_u32(&ctl.s_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.s_empty[b]), 4); }
-    sm100::mbar_init(sm100::smem_u32(&ctl.p_full), 4); sm100::mbar_init(sm100::smem_u32(&ctl.p_empty), 1);
+    for (int s = 0; s < K_STAGES; ++s) { sm100::mbar_init(sm100::smem_u32(&ctl.k_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.k_empty[s]), 1); }
+    for (int s = 0; s < V_STAGES; ++s) { sm100::mbar_init(sm100::smem_u32(&ctl.v_full[s]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.v_empty[s]), 1); }
+    for (int b = 0; b < 2; ++b) { sm100::mbar_init(sm100::smem_u32(&ctl.s_full[b]), 1); sm100::mbar_init(sm100::smem_u32(&ctl.s_empty[b]), 1); }
+    for (int b = 0; b < 2; ++b) sm100::mbar_init(sm100::smem_u32(&ctl.p_full[b]), 4);
     sm100::fence_mbar_init();
   }
   if (warp == 1) {
@@ -165,28 +164,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       sm100::mbar_expect_tx(qb, (uint32_t)(NH * rows_used * 128));
       for (int h = 0; h < NH; ++h)
         sm100::tma_load_3d(smem0 + L::Q_OFF + h * (128 * 128), &tmQ, qb, h * 64, kvh * a.G, row0, pol);
-      int s = 0; uint32_t ph = 0; bool ok = true;
-      for (int t = t_begin; t < t_end && ok; ++t) {
+      int ks = 0, vs = 0; uint32_t kph = 0, vph = 0;
+      auto load_tile = [&](int t, bool is_k) -> bool {
         const bool is_cache = t < n_cache_tiles;
         const int page = is_cache ? a.page_table[(size_t)seq * a.pages_per_seq + t] : 0;
         const int lrow = loc_lo + (t - n_cache_tiles) * KT;
-        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.k_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
-        uint32_t fb = sm100::smem_u32(&ctl.k_full[s]);
+        const int st = is_k ? ks : vs;
+        if (!sm100::mbar_wait(sm100::smem_u32(is_k ? &ctl.k_empty[st] : &ctl.v_empty[st]), (is_k ? kph : vph) ^ 1u, abortp)) return false;
+        const uint32_t fb = sm100::smem_u32(is_k ? &ctl.k_full[st] : &ctl.v_full[st]);
         sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
         for (int h = 0; h < NH; ++h) {
-          const uint32_t dst = smem0 + L::K_OFF + s * L::KV_BYTES + h * (KT * 128);
-          if (is_cache) sm100::tma_load_4d(dst, &tmK, fb, h * 64, 0, kvh, a.page_base_k + page, pol);
-          else sm100::tma_load_3d(dst, &tmKloc, fb, h * 64, kvh, lrow, pol);
+          const uint32_t dst = smem0 + (is_k ? L::K_OFF : L::V_OFF) + st * L::KV_BYTES + h * (KT * 128);
+          if (is_cache) sm100::tma_load_4d(dst, is_k ? &tmK : &tmV, fb, h * 64, 0, kvh, (is_k ? a.page_base_k : a.page_base_v) + page, pol);
+          else sm100::tma_load_3d(dst, is_k ? &tmKloc : &tmVloc, fb, h * 64, kvh, lrow, pol);
         }
-        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.v_empty[s]), ph ^ 1u, abortp)) { ok = false; break; }
-        fb = sm100::smem_u32(&ctl.v_full[s]);
-        sm100::mbar_expect_tx(fb, (uint32_t)L::KV_BYTES);
-        for (int h = 0; h < NH; ++h) {
-          const uint32_t dst = smem0 + L::V_OFF + s * L::KV_BYTES + h * (KT * 128);
-          if (is_cache) sm100::tma_load_4d(dst, &tmV, fb, h * 64, 0, kvh, a.page_base_v + page, pol);
-          else sm100::tma_load_3d(dst, &tmVloc, fb, h * 64, kvh, lrow, pol);
-        }
-        if (++s == KV_STAGES) { s = 0; ph ^= 1u; }
+        if (is_k) { if (++ks == K_STAGES) { ks = 0; kph ^= 1u; } }
+        else { if (++vs == V_STAGES) { vs = 0; vph ^= 1u; } }
+        return true;
+      };
+      // K of tile t + 1 goes out before V of tile t, in the order the MMA warp consumes them
+      bool ok = load_tile(t_begin, true);
+      for (int t = t_begin; t < t_end && ok; ++t) {
+        if (t + 1 < t_end) ok = load_tile(t + 1, true);
+        if (ok) ok = load_tile(t, false);
       }
     }
   } else if (warp == 1) {
@@ -201,7 +201,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       // descriptors are built once; the issue loop only adds 16-byte-unit offsets
       const uint64_t q_desc = sm100::make_desc_sw128(smem0 + L::Q_OFF);
       const uint64_t k_desc0 = sm100::make_desc_sw128(smem0 + L::K_OFF);
-      const uint64_t p_desc = sm100::make_desc_sw128(smem0 + L::P_OFF);
       const uint64_t v_desc0 = sm100::make_desc_sw128_mn(smem0 + L::V_OFF, KT * 128);
       constexpr uint64_t KV16 = L::KV_BYTES >> 4;
       auto issue_qk = [&](int i) -> bool {   // i: tile counter of this CTA
@@ -219,22 +218,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         sm100::mma_commit(sm100::smem_u32(&ctl.k_empty[ks]));
         sm100::mma_commit(sm100::smem_u32(&ctl.s_full[b]));
-        if (++ks == KV_STAGES) { ks = 0; kph ^= 1u; }
+        if (++ks == K_STAGES) { ks = 0; kph ^= 1u; }
         return true;
       };
       if (ok) ok = issue_qk(0);
       for (int i = 0; i < nt && ok; ++i) {
         if (i + 1 < nt) { ok = issue_qk(i + 1); if (!ok) break; }
         if (!sm100::mbar_wait(sm100::smem_u32(&ctl.v_full[vs]), vph, abortp)) { ok = false; break; }
-        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.p_full), (uint32_t)i & 1u, abortp)) { ok = false; break; }
+        // (one barrier per S buffer: the softmax warps may finish tile i + 1 before this thread has seen tile i,
+        // and a parity wait cannot tell two completions from none)
+        if (!sm100::mbar_wait(sm100::smem_u32(&ctl.p_full[i & 1]), (uint32_t)(i >> 1) & 1u, abortp)) { ok = false; break; }
         sm100::tc_fence_after();
         const uint64_t vd = v_desc0 + (uint64_t)vs * KV16;
+        const uint32_t p_tmem = tmem_S + (uint32_t)((i & 1) * KT);
 #pragma unroll
-        for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per instruction: 32 B along a P row, 16 V rows (2048 B)
-          sm100::mma_bf16_ss(tmem_O, p_desc + kk * 2, vd + kk * (16 * 128 / 16), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < KT / 16; ++kk)       // 16 keys per instruction: 8 columns of P, 16 V rows (2048 B)
+          sm100::mma_bf16_ts(tmem_O, p_tmem + kk * 8, vd + kk * (16 * 128 / 16), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         sm100::mma_commit(sm100::smem_u32(&ctl.v_empty[vs]));
-        sm100::mma_commit(sm100::smem_u32(&ctl.p_empty));      // P consumed and O up to date through tile i
-        if (++vs == KV_STAGES) { vs = 0; vph ^= 1u; }
+        // P consumed and O up to date through tile i: the S buffer P lived in is free for tile i + 2
+        sm100::mma_commit(sm100::smem_u32(&ctl.s_empty[i & 1]));
+        if (++vs == V_STAGES) { vs = 0; vph ^= 1u; }
       }
     }
   } else {
@@ -257,9 +260,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
         for (int j = 0; j < 32; ++j) { sv[j] = v0[j]; sv[32 + j] = v1[j]; }
       }
-      sm100::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&ctl.s_empty[b]));
 
       // visible keys of this tile for my row: [lo, hi) in tile-local indices
       int lo = 0, hi = 0;
@@ -309,9 +309,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       l_run = l_run * alpha + sum;
       m_ref = m_new;
 
-      // PV of the previous tile must be complete: it read P and updated O
-      if (!__all_sync(0xffffffffu, sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), ((uint32_t)i & 1u) ^ 1u, abortp))) { ok = false; break; }
       if (i > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        // O is rescaled in place, so P V of tile i - 1 must be complete: completion (i - 1) / 2 of the
+        // barrier of its S buffer.  A parity wait means what it says only while the barrier is at most
+        // one completion away from the one waited for, which holds although most tiles never wait
+        // here: completion (i - 3) / 2 happened before the Q K^T of tile i - 1 was issued, and the
+        // next one needs the P of tile i + 1.
+        if (!__all_sync(0xffffffffu, sm100::mbar_wait(sm100::smem_u32(&ctl.s_empty[(i - 1) & 1]), (uint32_t)((i - 1) >> 1) & 1u, abortp))) { ok = false; break; }
         sm100::tc_fence_after();
 #pragma unroll
         for (int c = 0; c < HD / 32; ++c) {
@@ -325,22 +329,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         sm100::tmem_wait_st();
         sm100::tc_fence_before();
       }
-      // P -> shared memory in the 128-byte-swizzled K-major operand layout
-      {
-        const uint32_t prow = smem0 + L::P_OFF + (my_row >> 3) * 1024 + (my_row & 7) * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint32_t dst = prow + ((c ^ (my_row & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pk[4 * c]), "r"(pk[4 * c + 1]), "r"(pk[4 * c + 2]),
-                       "r"(pk[4 * c + 3]) : "memory");
-        }
-      }
-      sm100::fence_proxy_async();
+      // P -> the first 32 columns of this tile's S buffer (my row = my TMEM lane; the scores are in registers)
+      sm100::tmem_st32(tmem_S + lane_addr + b * KT, pk);
+      sm100::tmem_wait_st();
+      sm100::tc_fence_before();
       __syncwarp();
-      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&ctl.p_full));
+      if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&ctl.p_full[b]));
     }
     // ---- output: O is complete once the last PV has finished ----
-    if (ok && nt > 0) ok = sm100::mbar_wait(sm100::smem_u32(&ctl.p_empty), (uint32_t)(nt - 1) & 1u, abortp);
+    // (the last two products, each on its own buffer's barrier; the bound on the distance holds as above)
+    if (ok && nt > 1) ok = sm100::mbar_wait(sm100::smem_u32(&ctl.s_empty[(nt - 2) & 1]), (uint32_t)((nt - 2) >> 1) & 1u, abortp);
+    if (ok && nt > 0) ok = sm100::mbar_wait(sm100::smem_u32(&ctl.s_empty[(nt - 1) & 1]), (uint32_t)((nt - 1) >> 1) & 1u, abortp);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       sm100::tc_fence_after();
