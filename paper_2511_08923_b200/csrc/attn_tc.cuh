@@ -20,7 +20,7 @@
 // V 16, and the 32 KB the TMA writes), 1000 cycles at 128 B per cycle against 512 cycles of MMAs.  The reference max is only raised when a tile
 // exceeds it by more than 2^8 (P stays <= 256, exact enough in bf16/fp32); raising it
 // rescales the rows of O in TMEM, which happens in the first tiles only.  The CTA needs
-// <= 97 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
+// <= 113 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
 // share an SM and fill each other's dependency stalls.  The key range of a query tile can be
 // split over several CTAs; partial (max, sum, O) results are merged by attn_combine_kernel.
 #pragma once
