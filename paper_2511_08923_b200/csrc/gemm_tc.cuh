@@ -294,16 +294,94 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         best_v[k] = -INFINITY; best_i[k] = 0x7fffffff;
       }
     };
+    // ---- MODE_SWIGLU: two 16-column chunks of the accumulator -> bf16 rows of H ----
+    // Lane pairs (2j, 2j+1) hold gate and up of feature n/2; the even lane finishes
+    // column c, the odd lane column c+1, after one exchange per column pair.  The
+    // results of a 16-column chunk (16 columns x 16 features per warp) are turned
+    // through shared memory so that every lane stores 8 consecutive features of one
+    // row with one 16-byte store: 2-byte stores from each lane took 18 us per tile.
+    // All exchanges first, then sixteen independent silu chains (one chain at a time is bound by
+    // instruction latency: 16 us per tile instead of 2), then the turn through shared memory.
+    // c0 / c1: the two chunks (c1 only if second); row0: output row of c0's first column.
+    auto swiglu_pass = [&](const uint32_t (&c0)[16], const uint32_t (&c1)[16], bool second, int row0, int R_live, int tile) {
+      const bool odd = lane & 1;
+      uint16_t (*stage)[16] = epi_stage[MODE == MODE_SWIGLU ? warp - ROLE_WARPS : 0];
+      const int srow = lane >> 1, sf = (lane & 1) * 8;
+      const int f0 = ((tile * TILE_N + q * 32) >> 1) + sf;          // first of this lane's 8 features
+      const int n_feat = g.N >> 1;
+      float h[2][8];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        if (c == 0 || second) {
+          uint32_t recv[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) recv[j] = __shfl_xor_sync(0xffffffffu, odd ? (c ? c1[2 * j] : c0[2 * j]) : (c ? c1[2 * j + 1] : c0[2 * j + 1]), 1);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float gate = __uint_as_float(odd ? recv[j] : (c ? c1[2 * j] : c0[2 * j]));
+            const float up = __uint_as_float(odd ? (c ? c1[2 * j + 1] : c0[2 * j + 1]) : recv[j]);
+            h[c][j] = silu_mul(gate, up);
+          }
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+        if (c == 0 || second) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) stage[c * 16 + 2 * j + (odd ? 1 : 0)][lane >> 1] = __bfloat16_as_ushort(__float2bfloat16(h[c][j]));
+        }
+      __syncwarp();
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+        if (c == 0 || second) {
+          const uint4 packed = *reinterpret_cast<const uint4 *>(&stage[c * 16 + srow][sf]);
+          const int r = row0 + c * 16 + srow;
+          if (r < R_live) {
+            bf16 *dst = g.H + (long long)r * g.ldh + f0;
+            if (f0 + 8 <= n_feat && (g.ldh & 7) == 0) {
+              *reinterpret_cast<uint4 *>(dst) = packed;
+            } else {
+              const uint16_t *e = reinterpret_cast<const uint16_t *>(&packed);
+              for (int t = 0; t < 8; ++t)
+                if (f0 + t < n_feat) dst[t] = __ushort_as_bfloat16(e[t]);
+            }
+          }
+        }
+      __syncwarp();
+    };
     // The epilogue below is long straight-line code that a CTA runs once or twice, and between two
     // launches of this kernel the other kernels of a layer push it out of the instruction cache: run
     // cold, next to the MMAs of the next item, one SwiGLU pass took 2 - 3.5 us instead of 0.4.  These
     // warps have nothing to do while the first item's MMAs run, so they first walk through the
     // epilogue once with every store and barrier operation switched off (dry), which
     // brings the code in; g.warm_epilogue is a run-time value so that both walks share one copy.
-    bool dry = (MODE == MODE_SWIGLU) && g.warm_epilogue != 0;
+    // A fused item that is its CTA's last one takes a third route: nobody waits for the accumulator, so it
+    // stays in tensor memory and a loop of a few hundred instructions takes 32 columns per round (the
+    // 1.5B-class gate/up projection, one item per CTA, ends 4 us earlier than with the long code).
+    bool dry = (MODE == MODE_SWIGLU) && g.warm_epilogue != 0 && (int)(blockIdx.x + gridDim.x) < n_items;
     for (int item = blockIdx.x; item < n_items && ok;) {
       const Item w = decode_item<MODE>(g, item);
       const int split = w.split, tile = w.tile, rb = w.rb;
+      if (MODE == MODE_SWIGLU && w.fused && item + (int)gridDim.x >= n_items) {
+        if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
+        sm100::tc_fence_after();
+        const uint32_t t0 = tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin;
+        const int row_first = rb * g.rb_rows + c_begin;
+#pragma unroll 1
+        for (int cc = 0; cc < ncols; cc += 32) {
+          uint32_t c0[16], c1[16];
+          const bool second = cc + 16 < ncols;
+          sm100::tmem_ld16(t0 + cc, c0);
+          if (second) sm100::tmem_ld16(t0 + cc + 16, c1);
+          sm100::tmem_wait_ld();
+          swiglu_pass(c0, c1, second, row_first + cc, g.R, tile);
+        }
+        sm100::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) sm100::mbar_arrive(sm100::smem_u32(&tmem_empty_bar));
+        item += gridDim.x; ++it;
+        continue;
+      }
       uint32_t v[9][16];
       if (!dry) {
         if (!sm100::mbar_wait(sm100::smem_u32(&tmem_full_bar), it & 1u, abortp)) { ok = false; break; }
@@ -365,63 +443,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
         }
       } else if (MODE == MODE_SWIGLU) {
-        // Lane pairs (2j, 2j+1) hold gate and up of feature n/2; the even lane finishes
-        // column c, the odd lane column c+1, after one exchange per column pair.  The
-        // results of a 16-column chunk (16 columns x 16 features per warp) are turned
-        // through shared memory so that every lane stores 8 consecutive features of one
-        // row with one 16-byte store: 2-byte stores from each lane took 18 us per tile.
-        const bool odd = lane & 1;
-        uint16_t (*stage)[16] = epi_stage[warp - ROLE_WARPS];
-        const int srow = lane >> 1, sf = (lane & 1) * 8;
-        const int f0 = ((tile * TILE_N + q * 32) >> 1) + sf;          // first of this lane's 8 features
-        const int n_feat = g.N >> 1;
-        // Two 16-column chunks per pass: all exchanges first, then sixteen independent silu
-        // chains (one chain at a time is bound by instruction latency: 16 us per tile instead of
-        // 2), then the turn through shared memory.
+        // Register-staged walk over the whole accumulator, two 16-column chunks per pass.
 #pragma unroll
         for (int ip = 0; ip < 5; ++ip) {
           if (ip * 32 < ncols) {
             const bool second = (2 * ip + 1) < 9 && (2 * ip + 1) * 16 < ncols;      // warp-uniform
-            float h[2][8];
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              const int i = (2 * ip + c) < 9 ? 2 * ip + c : 8;
-              if (c == 0 || second) {
-                uint32_t recv[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) recv[j] = __shfl_xor_sync(0xffffffffu, odd ? v[i][2 * j] : v[i][2 * j + 1], 1);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float gate = __uint_as_float(odd ? recv[j] : v[i][2 * j]);
-                  const float up = __uint_as_float(odd ? v[i][2 * j + 1] : recv[j]);
-                  h[c][j] = silu_mul(gate, up);
-                }
-              }
-            }
-#pragma unroll
-            for (int c = 0; c < 2; ++c)
-              if (c == 0 || second) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) stage[c * 16 + 2 * j + (odd ? 1 : 0)][lane >> 1] = __bfloat16_as_ushort(__float2bfloat16(h[c][j]));
-              }
-            __syncwarp();
-#pragma unroll
-            for (int c = 0; c < 2; ++c)
-              if (c == 0 || second) {
-                const uint4 packed = *reinterpret_cast<const uint4 *>(&stage[c * 16 + srow][sf]);
-                const int r = r_base + (2 * ip + c) * 16 + srow;
-                if (r < R_live) {
-                  bf16 *dst = g.H + (long long)r * g.ldh + f0;
-                  if (f0 + 8 <= n_feat && (g.ldh & 7) == 0) {
-                    *reinterpret_cast<uint4 *>(dst) = packed;
-                  } else {
-                    const uint16_t *e = reinterpret_cast<const uint16_t *>(&packed);
-                    for (int t = 0; t < 8; ++t)
-                      if (f0 + t < n_feat) dst[t] = __ushort_as_bfloat16(e[t]);
-                  }
-                }
-              }
-            __syncwarp();
+            swiglu_pass(v[2 * ip], v[(2 * ip + 1) < 9 ? 2 * ip + 1 : 8], second, r_base + ip * 32, R_live, tile);
           }
         }
       } else {
