@@ -592,9 +592,9 @@ DEFAULT_IMPL = 0
 # summarised in profiles/ (2-layer twin of the workload; per-layer traffic x n_layers + the LM
 # head launch).  Removed whenever the kernel changes after the capture.
 TRAFFIC = {
-    "8b": {"bytes_per_step": 36 * (111.2e6 + 53.6e6 + 35.9e6 + 208.1e6) + 1251.7e6,
-           "note": "ncu dram read+write per launch on the 2-layer twin (down 111.2, QKV 53.6, O 35.9, gate/up 208.1 MB; LM head "
-                   "1251.7 MB), x 36 layers + LM head; see profiles/gemm_tc_kernel_8b_shapes_R272.md"},
+    "8b": {"bytes_per_step": 36 * (111.0e6 + 53.6e6 + 35.9e6 + 208.6e6) + 1252.3e6,
+           "note": "ncu dram read+write per launch on the 2-layer twin (down 111.0, QKV 53.6, O 35.9, gate/up 208.6 MB; LM head "
+                   "1252.3 MB), x 36 layers + LM head; see profiles/gemm_tc_kernel_8b_shapes_R272.md"},
 }
 
 if __name__ == "__main__":
