@@ -154,10 +154,15 @@ int tidar_step(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_
                const int32_t *forced_accept /*host,[n_seqs] or NULL*/,
                int32_t *out_tokens /*host,[n_seqs][k_max]*/, int32_t *out_n /*host,[n_seqs]*/);
 
-/* Same as tidar_step but returns after enqueueing; results are fetched (and the
- * stream synchronised) by tidar_step_wait.  Used to time steps back to back.
- * Forced acceptance lengths are required (the host must know every sequence's
- * length to check capacity without reading the device).                           */
+/* Same as tidar_step but returns after enqueueing; tidar_step_wait blocks until the OLDEST
+ * enqueued step has finished and hands out its results.  Forced acceptance lengths are
+ * required (the host must know every sequence's length to check capacity without reading
+ * the device); the sequences' lengths are advanced when the step is enqueued.  A second step
+ * may be enqueued while the first is still in flight (two at most), so that the device never
+ * waits for the host between steps; a third, or a second one when per-step diagnostics are on
+ * (debug bits 0 / 3, timing, timeline), returns TIDAR_EINVAL.  Every other entry point that
+ * touches sequences returns TIDAR_EINVAL while a step is in flight.  If a step reports
+ * TIDAR_EDEVICE_TIMEOUT, the sequences of the step behind it are released as well.          */
 int tidar_step_async(tidar_ctx *ctx, const int32_t *seqs, int32_t n_seqs, const int32_t *forced_accept);
 int tidar_step_wait(tidar_ctx *ctx, int32_t *out_tokens /*host,[n_seqs][k_max]*/, int32_t *out_n /*host*/);
 

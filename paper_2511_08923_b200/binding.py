@@ -144,6 +144,7 @@ class Tidar:
                  guard_bytes: int = 0, beta: float = 1.0, prefill_rows: int = 0, temperature: float = 0.0, sample_seed: int = 0):
         self.lib = load()
         self.shape, self.k_max, self.max_batch = shape, k_max, max_batch
+        self._async_n = []                   # listed sequences of the steps in flight, oldest first
         self.device = torch.device(device)
         cfg = tidar_config(
             n_layers=len(packed["layers"]), d_model=shape.d_model, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
@@ -268,15 +269,19 @@ class Tidar:
         return out
 
     def step_async(self, seqs: Sequence[int], forced: Sequence[int]):
+        """Enqueues a step and returns; up to two may be in flight (see tidar_step_async)."""
         s, f = _i32(seqs), _i32(forced)
-        self._n_async = len(s)
         self._check(self.lib.tidar_step_async(self.ctx, _ip(s), len(s), _ip(f)))
+        self._async_n.append(len(s))
 
     def step_wait(self):
-        toks = np.empty((self._n_async, self.k_max), dtype=np.int32)
-        n = np.empty(self._n_async, dtype=np.int32)
+        """Results of the oldest step in flight (see tidar_step_wait)."""
+        m = self._async_n[0] if self._async_n else self.max_batch
+        toks = np.empty((m, self.k_max), dtype=np.int32)
+        n = np.empty(m, dtype=np.int32)
         self._check(self.lib.tidar_step_wait(self.ctx, _ip(toks), _ip(n)))
-        return [toks[i, :n[i]].tolist() for i in range(self._n_async)], n.tolist()
+        self._async_n.pop(0)
+        return [toks[i, :n[i]].tolist() for i in range(m)], n.tolist()
 
     def seq_len(self, seq: int) -> int:
         rc = self.lib.tidar_seq_len(self.ctx, seq)

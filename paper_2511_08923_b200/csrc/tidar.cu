@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <deque>
 #include <vector>
 
 #include "common.cuh"
@@ -55,7 +56,6 @@ struct tidar_ctx {
   int32_t *h_lay = nullptr;        // pinned staging for those five arrays
   size_t lay_ints = 0;
   int mixed_tiles = 0;             // query tiles of the current mixed step
-  std::vector<int> pending_ks;
   float *d_run_max = nullptr, *d_run_sum = nullptr, *d_tgt_logit = nullptr, *d_logprob = nullptr;   // likelihood scoring, per row
   int32_t *d_target = nullptr;
   std::vector<CUtensorMap> tm_lm_chunks;   // the LM head in vocabulary chunks of lm_chunk rows (scoring)
@@ -68,12 +68,19 @@ struct tidar_ctx {
   std::vector<SeqState> seqs;
   std::vector<int> free_pages;
   int32_t *h_pinned = nullptr;     // [max_batch*(k_max+1)] results + staging
-  int32_t *h_stage = nullptr;      // [2*max_batch] seq list + forced, pinned
   std::string err;
   int64_t launches = 0;
   // last pass
   int last_rows = 0, last_first_pos = 0;
-  std::vector<int> pending_seqs; std::vector<int> pending_forced; bool pending = false; int pending_k = 0;
+  // Steps that have been enqueued and not yet waited for, oldest first.  Two may be in flight when every
+  // acceptance length is forced (the host then knows the lengths without reading the device): the second
+  // is enqueued while the first runs, so the device never waits for the host between steps.
+  struct Flight { std::vector<int> seqs, ks; int k = 0, slot = 0; bool counted = false; };
+  std::deque<Flight> inflight;
+  cudaEvent_t flight_done[2] = {nullptr, nullptr};
+  int32_t *h_out2[2] = {nullptr, nullptr}, *h_stage2[2] = {nullptr, nullptr}, *h_status2[2] = {nullptr, nullptr};   // pinned, one set per slot
+  int32_t *h_page_table = nullptr;   // pinned mirror of the page table: the source of its (asynchronous) updates
+  int next_slot = 0;
   // tensor-core path
   gemm_tc::EncodeTiledFn encode = nullptr;
   std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wdown;
@@ -89,7 +96,6 @@ struct tidar_ctx {
   bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
   float *cand_val = nullptr;
-  int32_t *h_status = nullptr;
   // in-kernel timeline (diagnostics): two words per launch of the last recorded step
   static constexpr int TL_MAX = 2048;
   unsigned long long *d_tl = nullptr;
@@ -678,19 +684,22 @@ int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
   const int need = (upto_positions + c->cfg.page_size - 1) / c->cfg.page_size;
   if (need > c->pages_per_seq) return fail(c, TIDAR_ECAPACITY, "sequence %d needs %d pages, limit %d", seq, need, c->pages_per_seq);
   if ((int)s.pages.size() >= need) return TIDAR_OK;
+  // The copy reads a pinned mirror that nothing else writes at these entries until the sequence is
+  // released and prefilled again (which only happens with no step in flight), so it needs no wait.
+  int32_t *row = c->h_page_table + (size_t)seq * c->pages_per_seq;
+  const int have = (int)s.pages.size();
   while ((int)s.pages.size() < need) {
     if (c->free_pages.empty()) return fail(c, TIDAR_ECAPACITY, "KV page pool exhausted");
+    row[s.pages.size()] = c->free_pages.back();
     s.pages.push_back(c->free_pages.back());
     c->free_pages.pop_back();
   }
-  CUDA_TRY(c, cudaMemcpyAsync(c->d_page_table + (size_t)seq * c->pages_per_seq, s.pages.data(), s.pages.size() * sizeof(int),
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_page_table + (size_t)seq * c->pages_per_seq + have, row + have, (size_t)(need - have) * sizeof(int),
                               cudaMemcpyHostToDevice, c->stream));
-  // the source vector may be reallocated by a later call: make the copy complete first
-  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return TIDAR_OK;
 }
 
-// Enqueues every operation of one decode step for the sequences staged in h_stage.
+// Enqueues the kernels of one decode step (its inputs are already in d_step_seqs / d_forced).
 // k: block length of this step; ar: plain autoregressive step (the causal section alone).
 // mixed_R > 0: the listed sequences use different block lengths (layout staged in h_lay, mixed_R rows in all).
 int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, int mixed_R = 0) {
@@ -706,8 +715,6 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, in
     c->tl_n = 0; c->tl_cls.clear();
     CUDA_TRY(c, cudaMemsetAsync(c->d_tl, 0, 2 * tidar_ctx::TL_MAX * sizeof(unsigned long long), c->stream));
   }
-  CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-  CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   {
     Launch l(c, TIDAR_TC_EMBED);
     launch_after(assemble_step_kernel, R, 256, 0, c->stream, c->meta, c->d_step_seqs, c->d_seq_len, c->d_block, c->d_blk_len, k, n_blocks, lay, cf.k_max,
@@ -727,8 +734,6 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, in
     launch_after(kv_commit_kernel, dim3(n_seqs, cf.n_layers), 128, 0, c->stream, c->d_step_seqs, c->d_step_n, c->d_step_L, c->d_seq_len, k, lay.k,
                (cf.debug >> 1) & 1, geom(c), c->kv, c->pool_stride, l.tl);
   }
-  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-  CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaGetLastError());
   return TIDAR_OK;
 }
@@ -745,7 +750,10 @@ int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, in
     tidar_ctx::StepGraph &sg = c->sg;
     if (!sg.exec || sg.k != k || sg.ar != ar || sg.n_seqs != n_seqs || sg.splits != splits || sg.timeline != c->timeline ||
         sg.mixed_R != mixed_R || sg.tiles != tiles) {
-      if (sg.exec) { cudaGraphExecDestroy(sg.exec); sg.exec = nullptr; }
+      if (sg.exec) {
+        if (!c->inflight.empty()) CUDA_TRY(c, cudaStreamSynchronize(c->stream));    // the old graph may still be running
+        cudaGraphExecDestroy(sg.exec); sg.exec = nullptr;
+      }
       const int64_t l0 = c->launches;
       cudaGraph_t graph = nullptr;
       int rc = TIDAR_OK;
@@ -774,12 +782,55 @@ int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, in
   return record_step(c, n_seqs, k, hint, ar, mixed_R);
 }
 
+// Whether one more step may be enqueued: always when none is in flight; behind a step in flight only when
+// every acceptance length of both is forced (the host then knows the lengths without reading the device),
+// both use one block length for all their sequences and nothing reads per-step diagnostics.
+bool may_enqueue(tidar_ctx *c, bool all_forced, bool mixed) {
+  if (c->inflight.empty()) return true;
+  if (c->inflight.size() >= 2 || !all_forced || mixed || c->timing || c->timeline || (c->cfg.debug & (1 | 8))) return false;
+  return c->inflight.front().counted && c->inflight.front().ks.empty();
+}
+
+// The step proper: its inputs from the slot's pinned staging, the kernels (replayed graph or plain
+// launches), its results into the slot's pinned buffers, and the event its waiter blocks on.
+int launch_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles, int slot) {
+  const tidar_config &cf = c->cfg;
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage2[slot], n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage2[slot] + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  if (int rc = replay_or_record_step(c, n_seqs, k, hint, ar, mixed_R, tiles)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_out2[slot], c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_status2[slot], c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaEventRecord(c->flight_done[slot], c->stream));
+  return TIDAR_OK;
+}
+
+// Book-keeping of an enqueued step.  With every length forced the host advances the sequences now.
+void push_flight(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, int k, const int32_t *ks, int slot) {
+  tidar_ctx::Flight f;
+  f.seqs.assign(seqs, seqs + n_seqs);
+  if (ks) f.ks.assign(ks, ks + n_seqs);
+  f.k = k; f.slot = slot;
+  f.counted = forced != nullptr;
+  for (int i = 0; i < n_seqs && f.counted; ++i) f.counted = forced[i] > 0;
+  if (f.counted)
+    for (int i = 0; i < n_seqs; ++i) { c->seqs[seqs[i]].n += forced[i]; c->seqs[seqs[i]].k = ks ? ks[i] : k; }
+  c->inflight.push_back(std::move(f));
+  c->next_slot ^= 1;
+}
+
 // k_step: block length of this step (0 = the one the sequences' last pass left, which must then be
 // the same for all of them); ar: plain autoregressive step (k_step is 1).
 int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *forced, bool need_forced, int k_step = 0, bool ar = false) {
   const tidar_config &cf = c->cfg;
   if (!seqs || n_seqs < 1 || n_seqs > cf.max_batch) return fail(c, TIDAR_EINVAL, "n_seqs must be in [1, max_batch]");
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is already in flight; call tidar_step_wait first");
+  {
+    bool all_forced = forced != nullptr;
+    for (int i = 0; i < n_seqs && all_forced; ++i) all_forced = forced[i] > 0;
+    if (!may_enqueue(c, all_forced && need_forced, false))
+      return fail(c, TIDAR_EINVAL, c->inflight.size() >= 2 ? "two steps are already in flight; call tidar_step_wait first"
+                                                            : "a step is in flight; call tidar_step_wait first (a second step can only follow with forced lengths, "
+                                                              "one block length per step and no per-step diagnostics)");
+  }
   if (k_step < 0 || k_step > cf.k_max) return fail(c, TIDAR_EINVAL, "block length %d outside [1, k_max = %d]", k_step, cf.k_max);
   int k = ar ? 1 : k_step;
   for (int i = 0; i < n_seqs; ++i) {
@@ -800,16 +851,14 @@ int enqueue_step(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int32_t *f
     if (rc) return rc;
   }
   const int T = ar ? 1 : k * (k + 1), R = n_seqs * T;
-  for (int i = 0; i < n_seqs; ++i) { c->h_stage[i] = seqs[i]; c->h_stage[cf.max_batch + i] = forced ? forced[i] : 0; }
+  const int slot = c->next_slot;
+  for (int i = 0; i < n_seqs; ++i) { c->h_stage2[slot][i] = seqs[i]; c->h_stage2[slot][cf.max_batch + i] = forced ? forced[i] : 0; }
   int min_n = 1 << 30;
   for (int i = 0; i < n_seqs; ++i) min_n = std::min(min_n, c->seqs[seqs[i]].n);
   const int hint = (min_n + k + 63) / 64;
   const int spt = 128 / (cf.n_q_heads / cf.n_kv_heads);          // slots per attention query tile
-  if (int rc = replay_or_record_step(c, n_seqs, k, hint, ar, 0, n_seqs * ((T + spt - 1) / spt))) return rc;
-  c->pending_k = k;
-  c->pending_ks.clear();
-  c->pending_seqs.assign(seqs, seqs + n_seqs);
-  c->pending = true;
+  if (int rc = launch_step(c, n_seqs, k, hint, ar, 0, n_seqs * ((T + spt - 1) / spt), slot)) return rc;
+  push_flight(c, seqs, n_seqs, forced, k, nullptr, slot);
   c->last_hidden_off = 0;
   c->last_rows = R + ((cf.beta < 1.0f && !ar) ? n_seqs * k : 0); c->last_first_pos = -1;      // the mixed rows follow the slots
   // the host tracks lengths without reading the device when L is forced
@@ -830,7 +879,7 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
     same = same && ks[i] == ks[0];
   }
   if (same) return enqueue_step(c, seqs, n_seqs, forced, false, ks[0], false);
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is already in flight; call tidar_step_wait first");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight; call tidar_step_wait first");
   if (cf.beta < 1.0f) return fail(c, TIDAR_EINVAL, "beta < 1 needs one block length for all sequences of a step");
   for (int i = 0; i < n_seqs; ++i) {
     const int q = seqs[i], k = ks[i];
@@ -845,6 +894,7 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
     if (int rc = ensure_pages(c, seqs[i], c->seqs[seqs[i]].n + ks[i])) return rc;
   const int mb = cf.max_batch, spt = 128 / (cf.n_q_heads / cf.n_kv_heads);
   int32_t *hk = c->h_lay, *hoff = hk + (mb + 1), *hloc = hoff + (mb + 1), *ht0 = hloc + (mb + 1), *hte = ht0 + (c->R_head + mb);
+  const int slot = c->next_slot;
   int R = 0, loc = 0, tiles = 0, min_nk = 1 << 30;
   for (int i = 0; i < n_seqs; ++i) {
     const int k = ks[i], T = k * (k + 1);
@@ -852,43 +902,49 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
     for (int r0 = R; r0 < R + T; r0 += spt) { ht0[tiles] = r0; hte[tiles] = R + T; ++tiles; }
     R += T; loc += k * k;
     min_nk = std::min(min_nk, c->seqs[seqs[i]].n + k);
-    c->h_stage[i] = seqs[i]; c->h_stage[mb + i] = forced ? forced[i] : 0;
+    c->h_stage2[slot][i] = seqs[i]; c->h_stage2[slot][mb + i] = forced ? forced[i] : 0;
   }
   hk[n_seqs] = 0; hoff[n_seqs] = R; hloc[n_seqs] = loc;
   c->mixed_tiles = tiles;
   // a mixed step's kernels take every per-sequence length from the staged layout: the nominal k is unused
-  if (int rc = replay_or_record_step(c, n_seqs, 0, (min_nk + 63) / 64, false, R, tiles)) return rc;
-  c->pending_k = 0;
-  c->pending_ks.assign(ks, ks + n_seqs);
-  c->pending_seqs.assign(seqs, seqs + n_seqs);
-  c->pending = true;
+  if (int rc = launch_step(c, n_seqs, 0, (min_nk + 63) / 64, false, R, tiles, slot)) return rc;
+  push_flight(c, seqs, n_seqs, forced, 0, ks, slot);
   c->last_hidden_off = 0;
   c->last_rows = R; c->last_first_pos = -1;
   return TIDAR_OK;
 }
 
+// Waits for the oldest step in flight and hands out its results.
 int finish_step(tidar_ctx *c, int32_t *out_tokens, int32_t *out_n) {
-  if (!c->pending) return fail(c, TIDAR_EINVAL, "no step in flight");
-  c->pending = false;
-  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (c->inflight.empty()) return fail(c, TIDAR_EINVAL, "no step in flight");
+  tidar_ctx::Flight f = std::move(c->inflight.front());
+  c->inflight.pop_front();
+  CUDA_TRY(c, cudaEventSynchronize(c->flight_done[f.slot]));
   if (c->timing) collect_timing(c);
   if (c->timeline) collect_timeline(c);
-  if (c->h_status[0]) {
+  if (c->h_status2[f.slot][0]) {
     // The step's kernels have already rewritten the device-side lengths and blocks of the listed
-    // sequences from invalid results: their state is lost.  Release them; a new first pass is needed.
-    const int st = c->h_status[0];
-    c->h_status[0] = 0; cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
-    for (int q : c->pending_seqs) release_sequence(c, q);
+    // sequences from invalid results: their state is lost, and so is that of a step enqueued behind
+    // it.  Release them all; a new first pass is needed.
+    const int st = c->h_status2[f.slot][0];
+    cudaStreamSynchronize(c->stream);
+    c->h_status2[0][0] = 0; c->h_status2[1][0] = 0; cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream);
+    for (int q : f.seqs) release_sequence(c, q);
+    for (auto &g : c->inflight) for (int q : g.seqs) release_sequence(c, q);
+    c->inflight.clear();
     return fail(c, TIDAR_EDEVICE_TIMEOUT, "a bounded device-side wait gave up during the step (status %d); its results are invalid and the "
                                           "listed sequences were released (prefill them again)", st);
   }
   const int km = c->cfg.k_max;
-  for (size_t i = 0; i < c->pending_seqs.size(); ++i) {
-    const int L = c->h_pinned[i * (km + 1)];
-    c->seqs[c->pending_seqs[i]].n += L;
-    c->seqs[c->pending_seqs[i]].k = c->pending_ks.empty() ? c->pending_k : c->pending_ks[i];   // entries of the block the step left
+  const int32_t *res = c->h_out2[f.slot];
+  for (size_t i = 0; i < f.seqs.size(); ++i) {
+    const int L = res[i * (km + 1)];
+    if (!f.counted) {
+      c->seqs[f.seqs[i]].n += L;
+      c->seqs[f.seqs[i]].k = f.ks.empty() ? f.k : f.ks[i];        // entries of the block the step left
+    }
     if (out_n) out_n[i] = L;
-    if (out_tokens) for (int j = 0; j < km; ++j) out_tokens[i * km + j] = j < L ? c->h_pinned[i * (km + 1) + 1 + j] : -1;
+    if (out_tokens) for (int j = 0; j < km; ++j) out_tokens[i * km + j] = j < L ? res[i * (km + 1) + 1 + j] : -1;
   }
   return TIDAR_OK;
 }
@@ -950,12 +1006,26 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
   for (int i = 0; i < c->n_pages; ++i) c->free_pages[i] = i;
   uint32_t st = 0x9e3779b9u;
   for (int i = c->n_pages - 1; i > 0; --i) { st = st * 1664525u + 1013904223u; std::swap(c->free_pages[i], c->free_pages[(st >> 8) % (i + 1)]); }
-  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, ((size_t)cfg->max_batch * (cfg->k_max + 1) + 2 * cfg->max_batch + 16 + c->lay_ints) * sizeof(int), cudaHostAllocDefault);
+  // one pinned block: first-pass result | per slot: step results, staged inputs, status | mixed-step layout | page-table mirror
+  const size_t n_out = (size_t)cfg->max_batch * (cfg->k_max + 1), n_stage = 2 * (size_t)cfg->max_batch, n_pt = (size_t)cfg->max_batch * c->pages_per_seq;
+  cudaError_t e = cudaHostAlloc((void **)&c->h_pinned, (n_out + 2 * (n_out + n_stage + 16) + c->lay_ints + n_pt) * sizeof(int), cudaHostAllocDefault);
   if (e != cudaSuccess) { delete c; return fail(nullptr, TIDAR_ECUDA, "cudaHostAlloc: %s", cudaGetErrorString(e)); }
-  c->h_stage = c->h_pinned + (size_t)cfg->max_batch * (cfg->k_max + 1);
-  c->h_status = c->h_stage + 2 * cfg->max_batch;
-  c->h_lay = c->h_status + 16;
-  c->h_status[0] = 0;
+  {
+    int32_t *p = c->h_pinned + n_out;
+    for (int sl = 0; sl < 2; ++sl) {
+      c->h_out2[sl] = p; p += n_out;
+      c->h_stage2[sl] = p; p += n_stage;
+      c->h_status2[sl] = p; p += 16;
+      c->h_status2[sl][0] = 0;
+    }
+    c->h_lay = p; p += c->lay_ints;
+    c->h_page_table = p;
+    std::memset(c->h_page_table, 0, n_pt * sizeof(int));
+  }
+  for (int sl = 0; sl < 2; ++sl)
+    if (cudaEventCreateWithFlags(&c->flight_done[sl], cudaEventDisableTiming) != cudaSuccess) {
+      cudaFreeHost(c->h_pinned); delete c; return fail(nullptr, TIDAR_ECUDA, "cudaEventCreate failed");
+    }
   e = cudaMemsetAsync(c->d_seq_len, 0, cfg->max_batch * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 64 * sizeof(int), c->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_page_table, 0, (size_t)cfg->max_batch * c->pages_per_seq * sizeof(int), c->stream);
@@ -968,7 +1038,7 @@ int tidar_init(const tidar_config *cfg, const tidar_weights *w, void *arena, siz
 int tidar_prefill(tidar_ctx *c, int32_t seq, const int32_t *prompt, int32_t n_prompt, int32_t k, int32_t *out_first) {
   if (!c) return TIDAR_EINVAL;
   const tidar_config &cf = c->cfg;
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight");
   if (seq < 0 || seq >= cf.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
   if (!prompt || n_prompt < 1) return fail(c, TIDAR_EINVAL, "empty prompt");
   if (k < 1 || k > cf.k_max) return fail(c, TIDAR_EINVAL, "k must be in [1, k_max]");
@@ -1089,7 +1159,7 @@ int tidar_plan_ks(int32_t n_seqs, int32_t k_max, int32_t row_budget, const int32
 
 int tidar_release(tidar_ctx *c, int32_t seq) {
   if (!c) return TIDAR_EINVAL;
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight");
   if (seq < 0 || seq >= c->cfg.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
   if (c->seqs[seq].active) release_sequence(c, seq);
   return TIDAR_OK;
@@ -1098,7 +1168,7 @@ int tidar_release(tidar_ctx *c, int32_t seq) {
 int tidar_score(tidar_ctx *c, int32_t seq, const int32_t *ids, int32_t n, float *logprobs) {
   if (!c) return TIDAR_EINVAL;
   const tidar_config &cf = c->cfg;
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight");
   if (seq < 0 || seq >= cf.max_batch) return fail(c, TIDAR_EINVAL, "seq %d out of range", seq);
   if (!ids || !logprobs || n < 2) return fail(c, TIDAR_EINVAL, "tidar_score needs at least two token ids");
   if (n > cf.max_seq_len) return fail(c, TIDAR_ECAPACITY, "%d tokens exceed max_seq_len %d", n, cf.max_seq_len);
@@ -1145,6 +1215,7 @@ int tidar_free(tidar_ctx *c) {
   cudaStreamSynchronize(c->stream);
   for (auto &t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
   if (c->sg.exec) cudaGraphExecDestroy(c->sg.exec);
+  for (int sl = 0; sl < 2; ++sl) if (c->flight_done[sl]) cudaEventDestroy(c->flight_done[sl]);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
   return TIDAR_OK;
@@ -1298,7 +1369,7 @@ int tidar_debug_get_timing(tidar_ctx *c, float *ms) {
 int tidar_gemm(tidar_ctx *c, const void *A, const void *W, int32_t R, int32_t N, int32_t K, int32_t splits, float *out) {
   if (!c) return TIDAR_EINVAL;
   if (!A || !W || !out) return fail(c, TIDAR_EINVAL, "null argument");
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight");
   if (R < 1 || N < 1 || K < 64 || K % 64) return fail(c, TIDAR_EINVAL, "R, N >= 1 and K a positive multiple of 64 required");
   if (((uintptr_t)A | (uintptr_t)W) % 16) return fail(c, TIDAR_EINVAL, "A and W must be 16-byte aligned");
   if (splits < 0 || splits > c->S_max) return fail(c, TIDAR_EINVAL, "splits must be in [0, %d]", c->S_max);
@@ -1336,7 +1407,7 @@ int tidar_attention(tidar_ctx *c, const void *q, const void *k_pages, const void
   if (k < 1 || k > c->cfg.k_max || n_seqs < 1 || n_seqs * k * (k + 1) > c->R_cap) return fail(c, TIDAR_EINVAL, "n_seqs * k(k+1) exceeds the context's row capacity");
   if (n_pages < 1 || pages_per_seq < 1) return fail(c, TIDAR_EINVAL, "n_pages and pages_per_seq must be positive");
   if ((long long)pages_per_seq * c->cfg.page_size < k) return fail(c, TIDAR_EINVAL, "the page table cannot back the k causal slots");
-  if (c->pending) return fail(c, TIDAR_EINVAL, "a step is in flight");
+  if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight");
   if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)k_local | (uintptr_t)v_local | (uintptr_t)out) % 16 ||
       ((uintptr_t)page_table | (uintptr_t)seq_len) % 4)
     return fail(c, TIDAR_EINVAL, "tensors must be 16-byte aligned (page_table and seq_len 4-byte)");

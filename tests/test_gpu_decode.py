@@ -430,3 +430,54 @@ def test_long_first_pass_in_one_chunk(tiny, impl):
     np.testing.assert_array_equal(outs[0][1][0][0], outs[1][1][0][0]); np.testing.assert_array_equal(outs[0][1][0][1], outs[1][1][0][1])
     if top1_margin(fo.logits[n - 1]) > MARGIN:
         assert outs[0][0] == outs[1][0] == c
+
+
+def test_two_steps_in_flight_match_one_at_a_time():
+    """tidar_step_async accepts a second step while the first is in flight (forced lengths): the results,
+    handed out oldest first, the blocks and the cached K/V are bit-identical to the same steps run one at a
+    time; a third step, a step without forced lengths behind one in flight, and every other entry point
+    are refused until the queue is drained."""
+    from paper_2511_08923_b200 import TidarError
+    sh, wt = make_model("tiny", tied=False)
+    k = sh.k
+    prompts = [prompt_ids(sh, n=sh.prompt_len - 3 * q, seed=sh.seed + q) for q in range(2)]
+    forced = [[2, 1], [k, 3], [1, 1], [3, k], [2, 2], [k, k], [1, 2]]
+    runs = {}
+    for tag in ("serial", "pipelined"):
+        t = _gpu(sh, wt, 0, k_max=k, debug=0, max_batch=2, max_seq_len=256)     # diagnostics off: they allow one step in flight only
+        for q, p in enumerate(prompts):
+            t.prefill(q, p, k)
+        res = []
+        if tag == "serial":
+            for f in forced:
+                res.append(t.step([0, 1], forced=f))
+        else:
+            t.step_async([0, 1], forced[0])
+            for f in forced[1:]:
+                t.step_async([0, 1], f)
+                if f is forced[1]:
+                    with pytest.raises(TidarError):
+                        t.step_async([0, 1], f)                   # a third step
+                    with pytest.raises(TidarError):
+                        t.prefill(0, prompts[0], k)               # anything else that touches sequences
+                    assert t.seq_len(0) == len(prompts[0]) + forced[0][0] + forced[1][0]      # lengths advance when a step is enqueued
+                res.append(t.step_wait())
+            res.append(t.step_wait())
+            with pytest.raises(TidarError):
+                t.step_wait()                                     # nothing left in flight
+            t.step_async([0, 1], [1, 1])
+            with pytest.raises(TidarError):
+                t.step([0, 1])                                    # unforced lengths cannot follow a step in flight
+            t.step_wait()
+            res.append(None)
+        n = [t.seq_len(q) for q in range(2)]
+        blocks = [t.get_block(q, k) for q in range(2)]
+        upto = [len(prompts[q]) + sum(f[q] for f in forced) for q in range(2)]
+        kv = [[t.kv(q, l, 0, upto[q]) for l in range(sh.n_layers)] for q in range(2)]
+        runs[tag] = (res[:len(forced)], upto, kv, blocks if tag == "serial" else None)
+        assert n[0] >= upto[0] and n[1] >= upto[1]
+        _close(t)
+    assert runs["serial"][0] == runs["pipelined"][0]
+    for q in range(2):
+        for (k0, v0), (k1, v1) in zip(runs["serial"][2][q], runs["pipelined"][2][q]):
+            np.testing.assert_array_equal(k0, k1); np.testing.assert_array_equal(v0, v1)
