@@ -17,9 +17,11 @@
 // K 64, P as the tensor-memory operand, V as the MN-major shared-memory operand) accumulates in
 // TMEM over all key tiles.  P never touches shared memory: with P staged there the kernel moved
 // 128 KB through shared memory per key tile (Q 32 and K 16 read by Q K^T, P 16 written and read,
-// V 16, and the 32 KB the TMA writes), 1000 cycles at 128 B per cycle against 512 cycles of MMAs.  The reference max is only raised when a tile
-// exceeds it by more than 2^8 (P stays <= 256, exact enough in bf16/fp32); raising it
-// rescales the rows of O in TMEM, which happens in the first tiles only.  The CTA needs
+// V 16, and the 32 KB the TMA writes), 1000 cycles at 128 B per cycle against 512 cycles of MMAs.
+// The reference max is only raised when a tile exceeds it by more than 2^8 (P stays <= 256,
+// exact enough in bf16/fp32); raising it rescales the rows of O in TMEM, which happens in the
+// first tiles only.  Barriers that either side can run ahead on exist once per S buffer (a
+// parity wait cannot tell two completions from none).  The CTA needs
 // <= 113 KB of shared memory, 256 TMEM columns and < 170 registers per thread, so two CTAs
 // share an SM and fill each other's dependency stalls.  The key range of a query tile can be
 // split over several CTAs; partial (max, sum, O) results are merged by attn_combine_kernel.
