@@ -94,6 +94,48 @@ def test_likelihood_scoring_matches_causal_log_softmax(tiny, impl):
         _close(t)
 
 
+def test_autoregressive_mode_at_the_benchmark_widths():
+    """The one-slot step and the scoring pass at the 8B-class widths (two layers, 8192-entry vocabulary so
+    that the oracle stays fast): one-row projections (a 16-row MMA block), 4096-wide rows, 32 / 8 heads.
+    Logits of every autoregressive step and the log-probabilities of a 300-token pass against the oracle."""
+    from dataclasses import replace as _r
+    from tidar_synth import CONFIGS as CONFIGS_, gen_model_weights as gen_model_weights_
+    sh = _r(CONFIGS_["8b"].reduced(2), vocab=8192)
+    wt = gen_model_weights_(sh)
+    cfg, w = oracle_cfg(sh), O.weights_to_f64(wt)
+    prompt = prompt_ids(sh, n=90)
+    n_new = 8
+    ar = O.ar_generate(cfg, w, prompt, n_new)
+    fo = O.causal_forward(cfg, w, list(prompt) + ar)
+    m = top1_margin(fo.logits[len(prompt) - 1:len(prompt) - 1 + n_new])
+    t = _gpu(sh, wt, 0, k_max=4, debug=1, max_seq_len=512)
+    first = t.prefill(0, prompt, 1)
+    if m[0] > MARGIN:
+        assert first == ar[0]
+    for i in range(n_new - 1):
+        t.set_block(0, [ar[i]])                     # teacher-forced with the oracle's tokens
+        nxt = t.ar_step([0])
+        n_rows, _ = t.last_rows()
+        assert n_rows == 1
+        check_rows(t.logits(0, 1), fo.logits[len(prompt) + i:len(prompt) + i + 1], f"AR step {i} logits")
+        if m[i + 1] > MARGIN:
+            assert nxt == [ar[i + 1]], (i, nxt, ar[i + 1])
+    _close(t)
+    rng = np.random.default_rng(11)
+    ids = rng.integers(0, sh.vocab - 1, 300)
+    lg = O.causal_forward(cfg, w, ids).logits[:-1]
+    lse = np.log(np.exp(lg - lg.max(-1, keepdims=True)).sum(-1)) + lg.max(-1)
+    want = lg[np.arange(len(ids) - 1), ids[1:]] - lse
+    t = _gpu(sh, wt, 0, k_max=4, max_seq_len=512)
+    got = t.score(0, ids)
+    # a log-probability is a logit minus a log-sum-exp, and the log-sum-exp moves by at most the largest
+    # logit error: twice the per-row logit bound of the full-width comparisons (check_rows)
+    bound = 2 * TOL_LOGITS * np.maximum(1.0, np.maximum(np.abs(lg).max(-1), 4 * np.sqrt((lg ** 2).mean(-1))))
+    assert (np.abs(got - want) <= bound).all(), (np.abs(got - want) / bound).max()
+    assert np.sqrt(((got - want) ** 2).mean()) <= 0.5 * TOL_LOGITS            # and far better on average
+    _close(t)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_block_length_chosen_per_step(tiny, impl):
     """tidar_step_k: shorter and longer blocks than the previous pass left.  Greedy TiDAR with beta = 1
