@@ -182,8 +182,8 @@ int tidar_step_k(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t 
  * the method ties the sequences of a batch to one length.  The pass has sum_i ks[i]*(ks[i]+1) token
  * slots, sequence after sequence.  Per sequence the results are those of tidar_step_k with that
  * sequence's length (same tokens; hidden states up to the rounding of a different row count).
- * forced_accept[i] in [0, ks[i]].  Equal lengths take tidar_step_k's path; different lengths need
- * beta == 1 (TIDAR_EINVAL otherwise).
+ * forced_accept[i] in [0, ks[i]].  Equal lengths take tidar_step_k's path.  With beta < 1 the mixed
+ * verification rows (one per verified position) follow the slots, sequence after sequence.
  * out_tokens / out_n as in tidar_step.                                                        */
 int tidar_step_ks(tidar_ctx *ctx, const int32_t *seqs /*host,[n_seqs]*/, int32_t n_seqs, const int32_t *ks /*host,[n_seqs]*/,
                   const int32_t *forced_accept /*host or NULL*/, int32_t *out_tokens /*host,[n_seqs][k_max]*/,

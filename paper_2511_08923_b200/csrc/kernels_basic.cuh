@@ -402,7 +402,9 @@ __global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const 
   const int32_t *ids = arg_ids + (lay.k ? (size_t)lay.off[s] : (size_t)s * T);
   int32_t *blk = block_ids + (size_t)seq * k_max;
   const int valid = blk_len[seq];
-  const int tgt = lane < k ? (tgt_ids ? tgt_ids[(size_t)s * k + lane] : ids[lane]) : -1;
+  size_t tgt0 = (size_t)s * k;                    // this sequence's first verification target among the mixed rows
+  if (lay.k && tgt_ids) { tgt0 = 0; for (int t = 0; t < s; ++t) tgt0 += lay.k[t]; }
+  const int tgt = lane < k ? (tgt_ids ? tgt_ids[tgt0 + lane] : ids[lane]) : -1;
   const int mine = lane < k ? (lane < valid ? blk[lane] : -2) : -2;
   const int prev_tgt = __shfl_up_sync(0xffffffffu, tgt, 1);
   const bool agree = lane == 0 || (lane < k && lane < valid && mine == prev_tgt);
@@ -428,15 +430,27 @@ __global__ void verify_select_kernel(const int32_t *__restrict__ arg_ids, const 
 // head's input, one extra input row per verified position, and the LM head's argmax of that row
 // is the argmax of the mixed logits.  Block i handles pair i:
 //   a = a0 + (i / k) * a_seq + (i % k) * a_j,  b likewise,  dst = dst0 + i.
+// With per-sequence block lengths (lay.k != null) pair i belongs to the sequence whose pairs
+// (one per verified position, k_s of them) contain it: a = off_s + j, b = off_s + k_s + j * k_s.
 __global__ void mix_rows_kernel(bf16 *__restrict__ A, int d, float beta, int k, int a0, int a_seq, int a_j, int b0, int b_seq, int b_j,
-                                int dst0, uint32_t *__restrict__ skey, TlSlot tl) {
+                                StepLayout lay, int dst0, uint32_t *__restrict__ skey, TlSlot tl) {
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x == 0) tl_go(tl);
-  const int i = blockIdx.x, s = i / k, j = i % k;
-  const bf16 *ra = A + (size_t)(a0 + s * a_seq + j * a_j) * d, *rb = A + (size_t)(b0 + s * b_seq + j * b_j) * d;
+  const int i = blockIdx.x;
+  int row_a, row_b;
+  if (lay.k) {
+    int s = 0, p = 0;
+    while (s + 1 < lay.n_seqs && i >= p + lay.k[s]) { p += lay.k[s]; ++s; }
+    const int ks = lay.k[s], j = i - p;
+    row_a = lay.off[s] + j; row_b = lay.off[s] + ks + j * ks;
+  } else {
+    const int s = i / k, j = i % k;
+    row_a = a0 + s * a_seq + j * a_j; row_b = b0 + s * b_seq + j * b_j;
+  }
+  const bf16 *ra = A + (size_t)row_a * d, *rb = A + (size_t)row_b * d;
   bf16 *ro = A + (size_t)(dst0 + i) * d;
-  if (skey && threadIdx.x == 0) skey[dst0 + i] = skey[a0 + s * a_seq + j * a_j];     // the mixed row predicts what row a predicts
+  if (skey && threadIdx.x == 0) skey[dst0 + i] = skey[row_a];     // the mixed row predicts what row a predicts
   for (int c = threadIdx.x * 2; c < d; c += blockDim.x * 2) {
     const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(ra + c));
     const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(rb + c));

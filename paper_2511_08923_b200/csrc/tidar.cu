@@ -91,7 +91,7 @@ struct tidar_ctx {
   float *attn_part_O = nullptr, *attn_part_ml = nullptr;
   int n_sms = 0;
   // the launches of one decode step as an executable graph, valid for one (k, n_seqs, attention split)
-  struct StepGraph { int k = 0, n_seqs = 0, splits = 0, mixed_R = 0, tiles = 0; bool ar = false, timeline = false; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
+  struct StepGraph { int k = 0, n_seqs = 0, splits = 0, mixed_R = 0, tiles = 0, mixed_K = 0; bool ar = false, timeline = false; cudaGraphExec_t exec = nullptr; int64_t launches = 0; } sg;
   bool graphs_ok = true;
   bool slab_bf16 = false;          // split-K partial sums of the step in bf16 instead of fp32 (config debug bit 2)
   int32_t *d_status = nullptr, *cand_idx = nullptr;
@@ -518,7 +518,7 @@ void launch_norm(tidar_ctx *c, int R, const float *partials, int S, size_t strid
 // The transformer stack over R assembled rows (metadata and X already filled).
 // with_head: run final norm + LM head + per-row argmax.
 // Extra LM-head input rows that mix two final-normed rows each (beta < 1; see mix_rows_kernel).
-struct MixRows { int n = 0, k = 1, a0 = 0, a_seq = 0, a_j = 0, b0 = 0, b_seq = 0, b_j = 0; };
+struct MixRows { int n = 0, k = 1, a0 = 0, a_seq = 0, a_j = 0, b0 = 0, b_seq = 0, b_j = 0; StepLayout lay{nullptr, nullptr, nullptr, 0}; };
 
 // head_row0: the LM head (with_head) runs on rows [head_row0, R) only, followed by the mixed rows; the
 // argmax ids and the logits dump are indexed from head_row0.
@@ -578,7 +578,7 @@ if (tc && c->slab_bf16)
                                 cudaMemcpyDeviceToDevice, c->stream));
   if (with_head && mix.n > 0) {            // rows R .. R + mix.n - 1 of the LM head's input
     Launch lm(c, TIDAR_TC_NORM);
-    launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, R,
+    launch_after(mix_rows_kernel, mix.n, 256, 0, c->stream, c->A, d, cf.beta, mix.k, mix.a0, mix.a_seq, mix.a_j, mix.b0, mix.b_seq, mix.b_j, mix.lay, R,
                  cf.temperature > 0.f ? c->meta.skey : (uint32_t *)nullptr, lm.tl);
     R += mix.n;
   }
@@ -702,7 +702,8 @@ int ensure_pages(tidar_ctx *c, int seq, int upto_positions) {
 // Enqueues the kernels of one decode step (its inputs are already in d_step_seqs / d_forced).
 // k: block length of this step; ar: plain autoregressive step (the causal section alone).
 // mixed_R > 0: the listed sequences use different block lengths (layout staged in h_lay, mixed_R rows in all).
-int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, int mixed_R = 0) {
+// mixed_K: the sum of those block lengths (= verified positions, one mixed row each when beta < 1).
+int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, int mixed_R = 0, int mixed_K = 0) {
   const tidar_config &cf = c->cfg;
   const int n_blocks = ar ? 0 : k;
   const int T = k * (n_blocks + 1), R = mixed_R > 0 ? mixed_R : n_seqs * T;
@@ -722,7 +723,10 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, in
   }
   // beta < 1: the verified prediction of causal slot j mixes its row with the first slot of block j
   MixRows mix;
-  if (cf.beta < 1.0f && !ar) { mix.n = n_seqs * k; mix.k = k; mix.a0 = 0; mix.a_seq = T; mix.a_j = 1; mix.b0 = k; mix.b_seq = T; mix.b_j = k; }
+  if (cf.beta < 1.0f && !ar) {
+    if (mixed_R > 0) { mix.n = mixed_K; mix.lay = lay; }
+    else { mix.n = n_seqs * k; mix.k = k; mix.a0 = 0; mix.a_seq = T; mix.a_j = 1; mix.b0 = k; mix.b_seq = T; mix.b_j = k; }
+  }
   if (int rc = forward_rows(c, R, true, mixed_R > 0 ? 0 : T, key_tiles_hint, mix)) return rc;
   {
     Launch l(c, TIDAR_TC_VERIFY);
@@ -743,13 +747,13 @@ int record_step(tidar_ctx *c, int n_seqs, int k, int key_tiles_hint, bool ar, in
 // for the grid sizes and the attention key split, so the step is captured once per (k, n_seqs,
 // rows, query tiles, split) and replayed.  Per-launch timing and the debug read-backs use plain
 // launches.  tiles: query tiles of the attention kernel per KV head.
-int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles) {
+int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles, int mixed_K = 0) {
   const tidar_config &cf = c->cfg;
   if (cf.impl == 0 && c->graphs_ok && !c->timing && !(cf.debug & (1 | 8))) {
     const int splits = attn_key_splits(c, tiles * cf.n_kv_heads, hint);
     tidar_ctx::StepGraph &sg = c->sg;
     if (!sg.exec || sg.k != k || sg.ar != ar || sg.n_seqs != n_seqs || sg.splits != splits || sg.timeline != c->timeline ||
-        sg.mixed_R != mixed_R || sg.tiles != tiles) {
+        sg.mixed_R != mixed_R || sg.tiles != tiles || sg.mixed_K != mixed_K) {
       if (sg.exec) {
         if (!c->inflight.empty()) CUDA_TRY(c, cudaStreamSynchronize(c->stream));    // the old graph may still be running
         cudaGraphExecDestroy(sg.exec); sg.exec = nullptr;
@@ -759,7 +763,7 @@ int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, in
       int rc = TIDAR_OK;
       cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
       if (e == cudaSuccess) {
-        rc = record_step(c, n_seqs, k, hint, ar, mixed_R);
+        rc = record_step(c, n_seqs, k, hint, ar, mixed_R, mixed_K);
         e = cudaStreamEndCapture(c->stream, &graph);
       }
       if (e == cudaSuccess && rc == TIDAR_OK && graph) e = cudaGraphInstantiate(&sg.exec, graph, 0);
@@ -768,7 +772,7 @@ int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, in
         cudaGetLastError();                         // capture is not available here: plain launches from now on
         sg.exec = nullptr; c->graphs_ok = false;
       } else {
-        sg.k = k; sg.ar = ar; sg.n_seqs = n_seqs; sg.splits = splits; sg.timeline = c->timeline; sg.mixed_R = mixed_R; sg.tiles = tiles;
+        sg.k = k; sg.ar = ar; sg.n_seqs = n_seqs; sg.splits = splits; sg.timeline = c->timeline; sg.mixed_R = mixed_R; sg.tiles = tiles; sg.mixed_K = mixed_K;
         sg.launches = c->launches - l0;
       }
       c->launches = l0;
@@ -779,7 +783,7 @@ int replay_or_record_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, in
       return TIDAR_OK;
     }
   }
-  return record_step(c, n_seqs, k, hint, ar, mixed_R);
+  return record_step(c, n_seqs, k, hint, ar, mixed_R, mixed_K);
 }
 
 // Whether one more step may be enqueued: always when none is in flight; behind a step in flight only when
@@ -793,11 +797,11 @@ bool may_enqueue(tidar_ctx *c, bool all_forced, bool mixed) {
 
 // The step proper: its inputs from the slot's pinned staging, the kernels (replayed graph or plain
 // launches), its results into the slot's pinned buffers, and the event its waiter blocks on.
-int launch_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles, int slot) {
+int launch_step(tidar_ctx *c, int n_seqs, int k, int hint, bool ar, int mixed_R, int tiles, int slot, int mixed_K = 0) {
   const tidar_config &cf = c->cfg;
   CUDA_TRY(c, cudaMemcpyAsync(c->d_step_seqs, c->h_stage2[slot], n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(c->d_forced, c->h_stage2[slot] + cf.max_batch, n_seqs * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-  if (int rc = replay_or_record_step(c, n_seqs, k, hint, ar, mixed_R, tiles)) return rc;
+  if (int rc = replay_or_record_step(c, n_seqs, k, hint, ar, mixed_R, tiles, mixed_K)) return rc;
   CUDA_TRY(c, cudaMemcpyAsync(c->h_out2[slot], c->d_out, (size_t)n_seqs * (cf.k_max + 1) * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(c->h_status2[slot], c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaEventRecord(c->flight_done[slot], c->stream));
@@ -880,7 +884,6 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
   }
   if (same) return enqueue_step(c, seqs, n_seqs, forced, false, ks[0], false);
   if (!c->inflight.empty()) return fail(c, TIDAR_EINVAL, "a step is in flight; call tidar_step_wait first");
-  if (cf.beta < 1.0f) return fail(c, TIDAR_EINVAL, "beta < 1 needs one block length for all sequences of a step");
   for (int i = 0; i < n_seqs; ++i) {
     const int q = seqs[i], k = ks[i];
     if (q < 0 || q >= cf.max_batch || !c->seqs[q].active) return fail(c, TIDAR_EINVAL, "sequence %d is not prefilled", q);
@@ -895,10 +898,10 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
   const int mb = cf.max_batch, spt = 128 / (cf.n_q_heads / cf.n_kv_heads);
   int32_t *hk = c->h_lay, *hoff = hk + (mb + 1), *hloc = hoff + (mb + 1), *ht0 = hloc + (mb + 1), *hte = ht0 + (c->R_head + mb);
   const int slot = c->next_slot;
-  int R = 0, loc = 0, tiles = 0, min_nk = 1 << 30;
+  int R = 0, loc = 0, tiles = 0, min_nk = 1 << 30, sum_k = 0;
   for (int i = 0; i < n_seqs; ++i) {
     const int k = ks[i], T = k * (k + 1);
-    hk[i] = k; hoff[i] = R; hloc[i] = loc;
+    hk[i] = k; hoff[i] = R; hloc[i] = loc; sum_k += k;
     for (int r0 = R; r0 < R + T; r0 += spt) { ht0[tiles] = r0; hte[tiles] = R + T; ++tiles; }
     R += T; loc += k * k;
     min_nk = std::min(min_nk, c->seqs[seqs[i]].n + k);
@@ -907,10 +910,11 @@ int enqueue_step_mixed(tidar_ctx *c, const int32_t *seqs, int n_seqs, const int3
   hk[n_seqs] = 0; hoff[n_seqs] = R; hloc[n_seqs] = loc;
   c->mixed_tiles = tiles;
   // a mixed step's kernels take every per-sequence length from the staged layout: the nominal k is unused
-  if (int rc = launch_step(c, n_seqs, 0, (min_nk + 63) / 64, false, R, tiles, slot)) return rc;
+  const int mixed_rows = cf.beta < 1.0f ? sum_k : 0;         // one mixed LM-head input row per verified position
+  if (int rc = launch_step(c, n_seqs, 0, (min_nk + 63) / 64, false, R, tiles, slot, mixed_rows)) return rc;
   push_flight(c, seqs, n_seqs, forced, 0, ks, slot);
   c->last_hidden_off = 0;
-  c->last_rows = R; c->last_first_pos = -1;
+  c->last_rows = R + mixed_rows; c->last_first_pos = -1;
   return TIDAR_OK;
 }
 

@@ -220,6 +220,51 @@ def test_block_length_per_sequence_within_one_step(tiny, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+def test_block_length_per_sequence_with_beta_mixing(tiny, impl):
+    """beta < 1 in a step of mixed block lengths: the mixed verification rows (one per verified position,
+    sequence after sequence) follow the slots; per sequence the mixed logits, the acceptance and the tokens
+    are those of the oracle's own step at that block length (paper Section 4.4.3)."""
+    sh, wt, cfg, w, prompt = tiny
+    beta = 0.5
+    cfg_b = replace(cfg, beta=beta)
+    ks = [3, 4, 2]
+    prompts = [prompt, prompt_ids(sh, n=sh.prompt_len - 4, seed=sh.seed + 5), prompt_ids(sh, n=sh.prompt_len + 6, seed=sh.seed + 6)]
+    t = _gpu(sh, wt, impl, k_max=4, debug=1, max_batch=3, max_seq_len=256, beta=beta)
+    states = []
+    for q, (p, k) in enumerate(zip(prompts, ks)):
+        t.prefill(q, p, k)
+        states.append(O.prefill(cfg_b, w, p, k)[0])
+    R = sum(k * (k + 1) for k in ks)
+    for step in range(3):
+        blocks = []
+        for q in range(3):
+            t.set_block(q, states[q].block)
+            blocks.append(states[q].block.copy())
+        outs = [O.step(cfg_b, w, states[q]) for q in range(3)]
+        toks, L = t.step_ks([0, 1, 2], ks)
+        n_rows, _ = t.last_rows()
+        assert n_rows == R + sum(ks)
+        lg = t.logits(0, n_rows)
+        ids = t.argmax(0, n_rows)
+        r0, m0 = 0, R
+        for q, k in enumerate(ks):
+            T = k * (k + 1)
+            fo = outs[q].fwd.logits
+            ref_mixed = beta * fo[:k] + (1 - beta) * fo[k:].reshape(k, k, -1)[:, 0, :]
+            assert np.abs(lg[r0:r0 + T] - fo).max() <= TOL_LOGITS
+            assert np.abs(lg[m0:m0 + k] - ref_mixed).max() <= TOL_LOGITS, (step, q)
+            tg = ids[m0:m0 + k]
+            L_ref = O.accept_length(blocks[q], tg)
+            assert L[q] == L_ref and toks[q] == [int(x) for x in blocks[q][1:L_ref]] + [int(tg[L_ref - 1])]
+            if top1_margin(ref_mixed).min() > MARGIN:
+                assert L[q] == outs[q].L and toks[q] == outs[q].emitted
+            r0 += T; m0 += k
+        if any(L[q] != outs[q].L for q in range(3)):
+            break                                   # a near-tie went the other way: the caches have parted
+    _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 def test_mixed_block_lengths_keep_the_autoregressive_continuation(tiny, impl):
     """With beta = 1 and greedy decoding every sequence of a mixed step still emits the model's
     autoregressive continuation, whatever lengths the steps choose (changing from step to step)."""
