@@ -516,3 +516,39 @@ def test_seeded_sampling_draws_what_the_oracle_draws(tiny, impl):
     agree = next((i for i, (a, b) in enumerate(zip(out, ar)) if a != b), 24)
     assert agree >= 12, (out, ar)        # identical up to a near-tie of two differently rounded passes
     _close(t)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_seeded_sampling_with_per_sequence_block_lengths(tiny, impl):
+    """temperature > 0 in a step of mixed block lengths: the draw of every row is keyed by its own sequence
+    slot and predicted position, so each row of the mixed pass equals the argmax of its tempered logits plus
+    the oracle's noise for (slot, position), whatever the neighbours' block lengths are."""
+    from paper_2511_08923_b200 import Tidar, pack_weights
+    sh, wt, cfg, w, prompt = tiny
+    temp, seed = 0.7, 91
+    ks = [2, 4, 3]
+    prompts = [prompt_ids(sh, n=sh.prompt_len + 2 * q, seed=sh.seed + 20 + q) for q in range(3)]
+    t = Tidar(sh, pack_weights(wt, "cuda:0"), k_max=4, max_batch=3, max_seq_len=256, debug=1, impl=impl, temperature=temp, sample_seed=seed,
+              guard_bytes=64 * 1024)
+    for q in range(3):
+        t.prefill(q, prompts[q], ks[q])
+    for step in range(3):
+        n_before = [t.seq_len(q) for q in range(3)]
+        toks, L = t.step_ks([0, 1, 2], ks)
+        n_rows, _ = t.last_rows()
+        lg = t.logits(0, n_rows).astype(np.float64)
+        ids = t.argmax(0, n_rows)
+        r0, checked = 0, 0
+        for q, k in enumerate(ks):
+            _, _, _, pos = O.slot_layout(n_before[q], k)
+            pred = np.concatenate([pos[:k] + 1, pos[k:]])          # a causal slot predicts the next position, a mask slot its own
+            T = k * (k + 1)
+            sc = np.stack([lg[r0 + r] / temp + O.gumbel_noise(seed, q, int(p), sh.vocab) for r, p in enumerate(pred)])
+            sure = top1_margin(sc) > 1e-3
+            np.testing.assert_array_equal(ids[r0:r0 + T][sure], sc.argmax(-1)[sure])
+            checked += int(sure.sum())
+            assert 1 <= L[q] <= k and t.seq_len(q) == n_before[q] + L[q]
+            r0 += T
+        assert checked >= 0.9 * n_rows
+    assert t.arena_guard_intact()
+    t.close()
