@@ -28,6 +28,8 @@
  *     not touch the arena while the context exists.
  *   - All work is enqueued on the CUDA stream given to tidar_init.  tidar_prefill
  *     and tidar_step synchronise that stream before they return the tokens.
+ *   - A context is not synchronised between host threads: one thread at a time may call
+ *     into it (different contexts are independent).
  *   - There is no CPU fallback: without a CUDA device tidar_init fails.
  */
 #ifndef TIDAR_H_
