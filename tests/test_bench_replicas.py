@@ -61,3 +61,30 @@ def test_reference_arm_only_rank0_works():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_pipelined_steps_keeps_two_in_flight_and_collects_every_result():
+    """bench.pipelined_steps against a fake context: never more than two steps enqueued and not yet waited
+    for, results handed back oldest first, nothing left in flight, every step's tokens counted."""
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class Fake:
+        def __init__(self):
+            self.queue, self.max_in_flight, self.order = [], 0, []
+
+        def step_async(self, seqs, forced):
+            self.queue.append(list(forced))
+            self.max_in_flight = max(self.max_in_flight, len(self.queue))
+            assert len(self.queue) <= 2
+
+        def step_wait(self):
+            f = self.queue.pop(0)
+            self.order.append(f)
+            return [[0] * x for x in f], f
+
+    for n in (0, 1, 2, 5):
+        t = Fake()
+        forced = [[1 + i % 3, 2] for i in range(n)]
+        assert bench.pipelined_steps(t, [0, 1], forced) == sum(sum(f) for f in forced)
+        assert t.queue == [] and t.order == forced and t.max_in_flight == min(n, 2)
